@@ -1,0 +1,419 @@
+"""CPU oracle for the SDVG hot path.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, fp64 NumPy statement of what the path computes: 3D-RoPE on q/k,
+block-causal attention of one block against the rolling KV cache, the ring
+commit with eviction, the worst-frame router with a forced rejection of block
+0, and the per-block speculative schedule that strings them together.  Nothing
+here is blocked, fused or tuned; library matmul/exp are used as single steps.
+
+Only tests, the smoke check and the bench's ``cpu_baseline`` leg may import
+this package.  It shares no code with the CUDA library and never imports it.
+
+bf16 tensors are ``numpy.uint16`` bit patterns, widened exactly to float64.
+Token layout of a block tensor is [tokens, heads, head_dim], tokens ordered
+frame-major, then grid row, then grid column.
+
+Pins (see tests): every function below is pinned by at least one independent
+check (dense-mask brute force, closed forms, invariants, hand-worked router
+and ring cases, the accept-rate convention and the cost identity implied by
+Table 1).  Parity unpinned: none.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+ROPE_THETA = 10000.0
+
+# --------------------------------------------------------------------------
+# bf16 <-> float
+# --------------------------------------------------------------------------
+
+
+def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to float64."""
+    b = np.asarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
+    b = np.asarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def f32_to_bf16(x: np.ndarray) -> np.ndarray:
+    """float32 -> bf16 bits, round to nearest even; NaN stays a quiet NaN."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    r = ((u + np.uint32(0x7FFF) + lsb) >> np.uint32(16)).astype(np.uint16)
+    nan = np.isnan(f)
+    if nan.any():
+        r = np.where(nan, ((u >> np.uint32(16)) | np.uint32(0x0040)).astype(np.uint16), r)
+    return r
+
+
+def f64_to_bf16(x: np.ndarray) -> np.ndarray:
+    """float64 -> bf16 bits through float32 (two RNE roundings; within 1 bf16 ulp of exact)."""
+    return f32_to_bf16(np.asarray(x, dtype=np.float64).astype(np.float32))
+
+
+# --------------------------------------------------------------------------
+# 3D RoPE  (Sec. 4.1 "KV caching via RoPE positional embeddings")
+# --------------------------------------------------------------------------
+
+
+def rope_axis_pairs(head_dim: int) -> tuple[int, int, int]:
+    """Number of rotated (even, odd) pairs owned by the frame / height / width axes.
+
+    Height and width each own floor(D/6) pairs, the frame axis the rest of the
+    D/2 pairs (D=128 -> 22/21/21, D=64 -> 12/10/10).
+    """
+    if head_dim <= 0 or head_dim % 2:
+        raise ValueError("head_dim must be a positive even number")
+    p_hw = head_dim // 6
+    return head_dim // 2 - 2 * p_hw, p_hw, p_hw
+
+
+def token_positions(tokens: int, grid: tuple[int, int, int], frame_offset: int) -> np.ndarray:
+    """[tokens, 3] integer (frame, row, column) positions, frame-major order."""
+    F, Hg, Wg = grid
+    if tokens != F * Hg * Wg:
+        raise ValueError("tokens != F*Hg*Wg")
+    n = np.arange(tokens, dtype=np.int64)
+    f = n // (Hg * Wg) + frame_offset
+    y = (n // Wg) % Hg
+    x = n % Wg
+    return np.stack([f, y, x], axis=1)
+
+
+def rope_angles(head_dim: int, pos: np.ndarray) -> np.ndarray:
+    """[tokens, D/2] fp64 rotation angles: pair i of an axis with P pairs turns by pos*theta^(-i/P)."""
+    pf, ph, pw = rope_axis_pairs(head_dim)
+    cols = []
+    for axis, P in enumerate((pf, ph, pw)):
+        i = np.arange(P, dtype=np.float64)
+        omega = ROPE_THETA ** (-(i / P))
+        cols.append(pos[:, axis:axis + 1].astype(np.float64) * omega[None, :])
+    return np.concatenate(cols, axis=1)
+
+
+def rope_ref(x_bits: np.ndarray, grid: tuple[int, int, int], frame_offset: int) -> np.ndarray:
+    """fp64 3D-RoPE of a [tokens, heads, D] bf16 tensor; returns float64 (not rounded).
+
+    Pair p is (x[2p], x[2p+1]) and turns counter-clockwise by its angle.
+    """
+    T, H, D = x_bits.shape
+    x = bf16_to_f64(x_bits)
+    a = rope_angles(D, token_positions(T, grid, frame_offset))       # [T, D/2]
+    c, s = np.cos(a)[:, None, :], np.sin(a)[:, None, :]
+    re, im = x[..., 0::2], x[..., 1::2]
+    out = np.empty_like(x)
+    out[..., 0::2] = re * c - im * s
+    out[..., 1::2] = re * s + im * c
+    return out
+
+
+def rope_table(head_dim: int, tab_frames: int, grid_h: int, grid_w: int) -> np.ndarray:
+    """fp32 (cos, sin) table, the shared numeric input of the bit-level RoPE.
+
+    Flat float32 array of (cos, sin) pairs: frame positions 0..tab_frames-1 by
+    P_f pairs, then grid rows 0..grid_h-1 by P_h pairs, then grid columns
+    0..grid_w-1 by P_w pairs.  Angles are formed and evaluated in fp64 and
+    rounded once to fp32.
+    """
+    pf, ph, pw = rope_axis_pairs(head_dim)
+    parts = []
+    for n_pos, P in ((tab_frames, pf), (grid_h, ph), (grid_w, pw)):
+        i = np.arange(P, dtype=np.float64)
+        omega = ROPE_THETA ** (-(i / P))
+        a = np.arange(n_pos, dtype=np.float64)[:, None] * omega[None, :]
+        parts.append(np.stack([np.cos(a), np.sin(a)], axis=-1).reshape(-1))
+    return np.concatenate(parts).astype(np.float32)
+
+
+def rope_bitspec(x_bits: np.ndarray, grid: tuple[int, int, int], frame_offset: int,
+                 table: np.ndarray, tab_frames: int) -> np.ndarray:
+    """Bit-level RoPE: the fp32 operation sequence that fixes the cache contents.
+
+    With (c, s) read from ``table``:  re' = fl(fl(re*c) - fl(im*s)),
+    im' = fl(fl(re*s) + fl(im*c)), every fl() one IEEE fp32 rounding, no fused
+    multiply-add, then round-to-nearest-even to bf16.  Returns bf16 bits.
+    """
+    T, H, D = x_bits.shape
+    F, Hg, Wg = grid
+    pf, ph, pw = rope_axis_pairs(D)
+    if frame_offset < 0 or frame_offset + F > tab_frames:
+        raise ValueError("frame positions outside the table")
+    tab = np.asarray(table, dtype=np.float32)
+    t_f = tab[:tab_frames * pf * 2].reshape(tab_frames, pf, 2)
+    t_h = tab[tab_frames * pf * 2: tab_frames * pf * 2 + Hg * ph * 2].reshape(Hg, ph, 2)
+    t_w = tab[tab_frames * pf * 2 + Hg * ph * 2:].reshape(Wg, pw, 2)
+    pos = token_positions(T, grid, frame_offset)
+    cs = np.concatenate([t_f[pos[:, 0]], t_h[pos[:, 1]], t_w[pos[:, 2]]], axis=1)  # [T, D/2, 2]
+    c = cs[:, None, :, 0]
+    s = cs[:, None, :, 1]
+    x = bf16_to_f32(x_bits)
+    re, im = x[..., 0::2], x[..., 1::2]
+    out = np.empty_like(x)
+    # numpy float32 ufuncs round every product and sum separately (no contraction)
+    out[..., 0::2] = (re * c).astype(np.float32) - (im * s).astype(np.float32)
+    out[..., 1::2] = (re * s).astype(np.float32) + (im * c).astype(np.float32)
+    return f32_to_bf16(out)
+
+
+# --------------------------------------------------------------------------
+# Block-causal attention over the rolling cache
+# --------------------------------------------------------------------------
+
+
+def visible_blocks(block_index: int, slots: int) -> list[int]:
+    """Earlier blocks block ``b`` may attend to: the last slots-1 blocks before it."""
+    return list(range(max(0, block_index - (slots - 1)), block_index))
+
+
+def attn_ref(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray, scale: float,
+             heads=None, rows=None, row_chunk: int = 1024):
+    """Softmax attention of query rows against ALL given keys, in fp64.
+
+    q [Tq, H, D], k/v [Lk, H, D] as bf16 bits (k already roped and rounded, as
+    the cache holds it).  For each head h and row i:
+      s_j = scale * <q_i, k_j>,  p_j = exp(s_j - max s) / sum,  o = sum_j p_j v_j,
+      lse = max s + ln(sum exp(s_j - max s)).
+    ``heads`` / ``rows`` restrict the evaluation to a subset (sampling at large
+    shapes).  Returns (o [len(rows), len(heads), D] fp64, lse [len(heads), len(rows)] fp64).
+    """
+    Tq, H, D = q_bits.shape
+    heads = list(range(H)) if heads is None else list(heads)
+    rows = np.arange(Tq) if rows is None else np.asarray(rows, dtype=np.int64)
+    o = np.empty((rows.size, len(heads), D), dtype=np.float64)
+    lse = np.empty((len(heads), rows.size), dtype=np.float64)
+    for hi, h in enumerate(heads):
+        kh = bf16_to_f64(k_bits[:, h, :])
+        vh = bf16_to_f64(v_bits[:, h, :])
+        for r0 in range(0, rows.size, row_chunk):
+            rr = rows[r0:r0 + row_chunk]
+            qh = bf16_to_f64(q_bits[rr, h, :])
+            s = (qh @ kh.T) * scale
+            m = s.max(axis=1, keepdims=True)
+            p = np.exp(s - m)
+            l = p.sum(axis=1, keepdims=True)
+            o[r0:r0 + rr.size, hi, :] = (p @ vh) / l
+            lse[hi, r0:r0 + rr.size] = (m + np.log(l))[:, 0]
+    return o, lse
+
+
+def dense_bruteforce(q_blocks, k_blocks, v_blocks, scale: float, slots: int):
+    """All blocks as ONE sequence with an explicit block-causal window mask (tiny inputs).
+
+    Key j is visible to query i iff blk(j) <= blk(i) and blk(i)-blk(j) <= slots-1.
+    Returns (o [B*T, H, D] fp64, P [H, B*T, B*T] fp64, mask [B*T, B*T] bool).
+    """
+    B = len(q_blocks)
+    T, H, D = q_blocks[0].shape
+    q = bf16_to_f64(np.concatenate(q_blocks, axis=0))
+    k = bf16_to_f64(np.concatenate(k_blocks, axis=0))
+    v = bf16_to_f64(np.concatenate(v_blocks, axis=0))
+    blk = np.repeat(np.arange(B), T)
+    mask = (blk[None, :] <= blk[:, None]) & ((blk[:, None] - blk[None, :]) <= slots - 1)
+    L = B * T
+    o = np.zeros((L, H, D))
+    P = np.zeros((H, L, L))
+    for h in range(H):
+        for i in range(L):
+            logits = np.full(L, -np.inf)
+            for j in range(L):
+                if mask[i, j]:
+                    logits[j] = scale * float(np.dot(q[i, h], k[j, h]))
+            e = np.exp(logits - logits.max())
+            P[h, i] = e / e.sum()
+            o[i, h] = P[h, i] @ v[:, h, :]
+    return o, P, mask
+
+
+# --------------------------------------------------------------------------
+# Ring KV cache (Sec. 3 "Inference flow": K^D updated always, K^T on accept / regenerate)
+# --------------------------------------------------------------------------
+
+STAGE = 1
+FINAL = 2
+
+
+class RingCacheRef:
+    """Integer model of the rolling cache: block b lives in slot b mod slots.
+
+    ``commit(b, k, v, FINAL)`` requires b == next_block, reports the block that
+    was evicted from the slot (-1 if it was empty) and advances next_block.
+    ``STAGE`` writes the bits of the provisional block b == next_block into its
+    slot (overwriting block b-slots, which b can no longer see) but leaves
+    next_block and the slot map alone.  Contents are exact copies of the input.
+    """
+
+    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int):
+        if min(slots, heads, block_tokens, head_dim) <= 0:
+            raise ValueError("bad cache shape")
+        self.slots, self.heads, self.T, self.D = slots, heads, block_tokens, head_dim
+        self.k = np.zeros((slots, block_tokens, heads, head_dim), dtype=np.uint16)
+        self.v = np.zeros_like(self.k)
+        self.next_block = 0
+        self.slot_block = [-1] * slots
+
+    def slot_of(self, block_index: int) -> int:
+        return block_index % self.slots
+
+    def commit(self, block_index: int, k_bits: np.ndarray, v_bits: np.ndarray, flags: int) -> int:
+        if flags not in (STAGE, FINAL):
+            raise ValueError("flags must be STAGE or FINAL")
+        if block_index != self.next_block:
+            raise RuntimeError("blocks must be committed in order")
+        if k_bits.shape != (self.T, self.heads, self.D) or v_bits.shape != k_bits.shape:
+            raise ValueError("bad block shape")
+        s = self.slot_of(block_index)
+        self.k[s] = k_bits
+        self.v[s] = v_bits
+        if flags == STAGE:
+            return -1
+        evicted = self.slot_block[s]
+        self.slot_block[s] = block_index
+        self.next_block = block_index + 1
+        return evicted
+
+    def window(self, block_index: int):
+        """Concatenated K, V ([n*T, H, D] bits) of the committed blocks visible to block_index."""
+        if block_index != self.next_block:
+            raise RuntimeError("attention is defined for the next block only")
+        ks, vs = [], []
+        for b in visible_blocks(block_index, self.slots):
+            s = self.slot_of(b)
+            if self.slot_block[s] != b:
+                raise RuntimeError("visible block is not in the ring")
+            ks.append(self.k[s])
+            vs.append(self.v[s])
+        if not ks:
+            e = np.zeros((0, self.heads, self.D), dtype=np.uint16)
+            return e, e.copy()
+        return np.concatenate(ks, axis=0), np.concatenate(vs, axis=0)
+
+
+def block_attn_ref(q_bits, k_self_bits, v_self_bits, cache: RingCacheRef, block_index: int,
+                   scale: float, heads=None, rows=None):
+    """Attention of block b: keys = visible committed blocks + the block itself, all visible."""
+    kw, vw = cache.window(block_index)
+    k_all = np.concatenate([kw, k_self_bits], axis=0)
+    v_all = np.concatenate([vw, v_self_bits], axis=0)
+    return attn_ref(q_bits, k_all, v_all, scale, heads=heads, rows=rows)
+
+
+# --------------------------------------------------------------------------
+# Router (Sec. 3: policy pi, Eq. (1) worst-frame aggregation, forced rejection of block 0)
+# --------------------------------------------------------------------------
+
+
+def route_ref(scores: np.ndarray, frame_offsets, num_blocks: int, frames_per_block: int,
+              first_block_index: int, tau: float):
+    """accept_b = (global block index != 0) and (min_i score[b, i] >= tau), in fp32.
+
+    ``scores`` is flat fp32; block b owns scores[frame_offsets[b]:frame_offsets[b+1]],
+    or frames_per_block consecutive values when frame_offsets is None.  The
+    minimum is taken left to right with a strict '<', so ties (and +0/-0) keep
+    the lowest index; any NaN frame makes q_min that NaN (lowest such index)
+    and the block is rejected.  Returns (accept u8[B], q_min f32[B], argmin i32[B]).
+    """
+    s = np.asarray(scores, dtype=np.float32).reshape(-1)
+    tau32 = np.float32(tau)
+    accept = np.zeros(num_blocks, dtype=np.uint8)
+    q_min = np.zeros(num_blocks, dtype=np.float32)
+    argmin = np.zeros(num_blocks, dtype=np.int32)
+    for b in range(num_blocks):
+        if frame_offsets is None:
+            lo, hi = b * frames_per_block, (b + 1) * frames_per_block
+        else:
+            lo, hi = int(frame_offsets[b]), int(frame_offsets[b + 1])
+        if hi <= lo:
+            raise ValueError("a block needs at least one frame")
+        m, idx = s[lo], 0
+        for i in range(lo + 1, hi):
+            x = s[i]
+            if np.isnan(m):
+                break
+            if np.isnan(x) or x < m:
+                m, idx = x, i - lo
+        q_min[b] = m
+        argmin[b] = idx
+        accept[b] = 1 if ((first_block_index + b) != 0 and (not np.isnan(m)) and m >= tau32) else 0
+    return accept, q_min, argmin
+
+
+def accept_rate(accept: np.ndarray, first_block_index: int = 0) -> float:
+    """Accept rate with block 0 left out of the count (convention of Tables 1 and 2)."""
+    a = np.asarray(accept).astype(np.int64)
+    idx = np.arange(a.size) + first_block_index
+    keep = idx != 0
+    return float(a[keep].sum()) / float(max(1, keep.sum()))
+
+
+# --------------------------------------------------------------------------
+# Per-block speculative schedule (Sec. 3 "Inference flow", Fig. 2)
+# --------------------------------------------------------------------------
+
+
+@dataclass
+class TraceResult:
+    accept: np.ndarray
+    q_min: np.ndarray
+    drafter_evicted: list = field(default_factory=list)
+    target_evicted: list = field(default_factory=list)
+    drafter_attn_calls: int = 0
+    target_attn_calls: int = 0
+    target_source: list = field(default_factory=list)   # per block: "accepted" or "regenerated"
+
+
+def schedule_ref(num_blocks: int, steps: int, scores: np.ndarray, tau: float,
+                 drafter: RingCacheRef, target: RingCacheRef, provider,
+                 grid_d, grid_t, frames_per_block_latent: int,
+                 tab_d, tab_t, tab_frames: int, on_attention=None) -> TraceResult:
+    """Run the per-block flow with the reference pieces.
+
+    For every block b: the drafter takes ``steps`` denoise steps (each: rope q,k
+    at frame offset b*frames -> stage k',v -> attention), then its clean K/V are
+    committed to the drafter ring unconditionally.  The router scores the block.
+    Accepted: the target-shaped K/V of the draft are committed to the target
+    ring.  Rejected (always block 0): the target takes ``steps`` steps of its
+    own and commits its clean K/V.  ``provider(model, block, kind, step)``
+    returns the (q, k, v) bf16 bits of that call (q is None for clean K/V).
+    ``on_attention(model, block, step, q_roped, k_roped, v, cache)`` lets a test
+    evaluate sampled attention rows at that point.
+    """
+    scores = np.asarray(scores, dtype=np.float32)
+    accept, q_min, _ = route_ref(scores.reshape(-1), None, num_blocks, scores.shape[1], 0, tau)
+    res = TraceResult(accept=accept, q_min=q_min)
+
+    def denoise(model, cache, grid, tab, b, kind):
+        calls = 0
+        for s in range(steps):
+            q, k, v = provider(model, b, kind, s)
+            fo = b * frames_per_block_latent
+            qr = rope_bitspec(q, grid, fo, tab, tab_frames)
+            kr = rope_bitspec(k, grid, fo, tab, tab_frames)
+            cache.commit(b, kr, v, STAGE)
+            if on_attention is not None:
+                on_attention(model, b, s, qr, kr, v, cache)
+            calls += 1
+        return calls
+
+    for b in range(num_blocks):
+        res.drafter_attn_calls += denoise("drafter", drafter, grid_d, tab_d, b, "step")
+        _, k, v = provider("drafter", b, "clean", 0)
+        kr = rope_bitspec(k, grid_d, b * frames_per_block_latent, tab_d, tab_frames)
+        res.drafter_evicted.append(drafter.commit(b, kr, v, FINAL))
+        if accept[b]:
+            _, k, v = provider("target", b, "accepted", 0)
+            res.target_source.append("accepted")
+        else:
+            res.target_attn_calls += denoise("target", target, grid_t, tab_t, b, "step")
+            _, k, v = provider("target", b, "clean", 0)
+            res.target_source.append("regenerated")
+        kr = rope_bitspec(k, grid_t, b * frames_per_block_latent, tab_t, tab_frames)
+        res.target_evicted.append(target.commit(b, kr, v, FINAL))
+    return res
