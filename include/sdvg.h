@@ -1,0 +1,214 @@
+/*
+ * sdvg.h — C ABI of the SDVG hot-path library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements what every drafter and target denoising step of SDVG
+ * (speculative decoding for block-autoregressive video diffusion) pays in its
+ * attention backbone (Sec. 4.1 "Models": causal attention with KV caching via
+ * RoPE, bf16) plus the routing rule of Sec. 3:
+ *
+ *   sdvg_rope3d_qk        3D rotary embedding (frame, row, column) of q and k
+ *   sdvg_block_attn_fwd   a block of latent frames attends to itself (all keys
+ *                         visible) and to the earlier blocks held in a rolling cache
+ *   sdvg_kv_commit        write a block's K/V into its ring slot, evicting the oldest
+ *   sdvg_route            worst-frame minimum against tau, block 0 always rejected
+ *
+ * Conventions
+ *   - Every function returns an int status (SDVG_OK == 0).  Nothing throws or
+ *     aborts.  All argument and state checks happen on the host before any
+ *     launch; a call that returns an error has enqueued nothing.
+ *   - "device" pointers are CUDA device memory owned by the caller; "host"
+ *     pointers are ordinary host memory.  The library allocates no device memory.
+ *   - bf16 tensors are [tokens, heads, head_dim], head_dim contiguous, tokens of
+ *     a block ordered frame-major, then grid row, then grid column.  All tensor
+ *     pointers must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Kernels are enqueued on it; the library never synchronises the device
+ *     unless a function says so.
+ *   - Functions that take a cache mutate only host metadata of that handle
+ *     besides enqueuing work; a handle must not be used from two threads at once.
+ */
+#ifndef SDVG_H_
+#define SDVG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------ */
+#define SDVG_OK                   0
+#define SDVG_ERR_INVALID_ARG      1   /* NULL pointer, negative size, unknown flag */
+#define SDVG_ERR_BAD_SHAPE        2   /* sizes inconsistent or unsupported (head_dim not 64/128, F=0, ...) */
+#define SDVG_ERR_MISALIGNED       3   /* a tensor pointer is not 16-byte aligned */
+#define SDVG_ERR_BAD_STATE        4   /* block out of order, self not staged, frame outside the table, ... */
+#define SDVG_ERR_UNSUPPORTED_ARCH 5   /* current device is not compute capability 10.x */
+#define SDVG_ERR_CUDA             6   /* a CUDA call failed: see sdvg_last_cuda_error() */
+#define SDVG_ERR_TIMEOUT          7   /* a bounded device-side wait gave up (reported by sdvg_block_attn_status) */
+
+/* ---- commit flags ------------------------------------------------------ */
+#define SDVG_STAGE 1   /* write the slot of the block being generated; ring state unchanged */
+#define SDVG_FINAL 2   /* write the slot, record the block as committed, advance to the next block */
+
+const char* sdvg_status_string(int status);
+/* Last cudaError_t seen by this thread inside the library (0 if none) and its text. */
+int         sdvg_last_cuda_error(void);
+const char* sdvg_last_cuda_error_string(void);
+
+/* ---- 3D RoPE ----------------------------------------------------------- */
+/*
+ * Pair split of the head dimension (Sec. 4.1 names RoPE only; the split is the
+ * Wan-family convention): height and width own floor(D/6) (even, odd) pairs
+ * each, the frame axis the remaining D/2 - 2*floor(D/6).  Pair i of an axis
+ * with P pairs rotates by position * 10000^(-i/P).
+ */
+int sdvg_rope3d_pairs(int head_dim, int* pairs_frame, int* pairs_height, int* pairs_width);
+
+/*
+ * (cos, sin) table in fp32, the numeric input that fixes RoPE results to the bit.
+ * Layout: for frame positions 0..tab_frames-1, P_f (cos, sin) pairs each; then
+ * for rows 0..grid_h-1, P_h pairs each; then for columns 0..grid_w-1, P_w pairs
+ * each.  Angles are formed and evaluated in fp64 and rounded once to fp32.
+ * sdvg_rope3d_table_floats returns the number of floats (0 on bad arguments);
+ * sdvg_rope3d_table fills a HOST buffer of that size.  The caller uploads it.
+ */
+size_t sdvg_rope3d_table_floats(int head_dim, int tab_frames, int grid_h, int grid_w);
+int    sdvg_rope3d_table(float* host_out, int head_dim, int tab_frames, int grid_h, int grid_w);
+
+/*
+ * Rotate q and k (device, bf16 [tokens, heads, head_dim]) into q_out, k_out
+ * (same layout; in-place allowed, q_out==q and/or k_out==k).  Either pair
+ * (q, q_out) or (k, k_out) may be NULL/NULL to rotate only one tensor.
+ * tokens must equal frames*grid_h*grid_w; token n sits at frame
+ * frame_offset + n/(grid_h*grid_w), row (n/grid_w)%grid_h, column n%grid_w.
+ * Arithmetic (per pair, c/s from the table): re' = fl(fl(re*c) - fl(im*s)),
+ * im' = fl(fl(re*s) + fl(im*c)) in IEEE fp32 without fused multiply-add,
+ * then round-to-nearest-even to bf16.
+ * cos_sin_tab: device copy of the table built for (head_dim, tab_frames, grid_h, grid_w).
+ * Errors: BAD_SHAPE (head_dim not 64/128, tokens mismatch), BAD_STATE
+ * (frame_offset < 0 or frame_offset+frames > tab_frames), MISALIGNED, INVALID_ARG.
+ */
+int sdvg_rope3d_qk(const void* q, const void* k, void* q_out, void* k_out,
+                   int tokens, int heads, int head_dim,
+                   int frames, int grid_h, int grid_w, int frame_offset,
+                   const float* cos_sin_tab, int tab_frames, void* stream);
+
+/* ---- rolling KV cache (Sec. 3 "Inference flow": K^D and K^T) ------------- */
+typedef struct sdvg_cache sdvg_cache;   /* opaque; owns host metadata only */
+
+/* Bytes of ONE buffer (K or V) for the given shape; 0 on bad arguments. */
+size_t sdvg_cache_bytes(int slots, int heads, int block_tokens, int head_dim);
+
+/*
+ * Bind a cache handle to two caller-owned device buffers of sdvg_cache_bytes()
+ * each, 1024-byte aligned.  Physical layout of each buffer (library's choice,
+ * readable through sdvg_cache_read_block): [heads][slots][block_tokens][head_dim]
+ * bf16, so that one head's ring is one contiguous run of keys.  Block b lives in
+ * slot b % slots.  slots = visible earlier blocks + 1.  The buffers are not
+ * cleared; empty slots are never read.
+ */
+int sdvg_cache_create(sdvg_cache** out, void* k_buf, void* v_buf,
+                      int slots, int heads, int block_tokens, int head_dim);
+int sdvg_cache_reset(sdvg_cache* cache);      /* forget all blocks (host state only) */
+int sdvg_cache_destroy(sdvg_cache* cache);    /* frees the handle, not the buffers */
+/*
+ * Host-side ring state: next block to be generated, slot -> committed block
+ * (-1 = empty; slot_block may be NULL or an array of `slots` entries) and the
+ * block currently staged (-1 if none; may be NULL).
+ */
+int sdvg_cache_state(const sdvg_cache* cache, int64_t* next_block, int64_t* slot_block,
+                     int64_t* staged_block);
+/* Gather one slot back into logical [block_tokens, heads, head_dim] device tensors (either may be NULL). */
+int sdvg_cache_read_block(const sdvg_cache* cache, int slot, void* k_out, void* v_out, void* stream);
+
+/*
+ * Commit (Sec. 3: the drafter cache is updated with every draft block; the
+ * target cache receives the accepted draft block or the regenerated one).
+ * Copies k_roped and v (device, bf16 [block_tokens, heads, head_dim]) into slot
+ * block_index % slots.  block_index must be the cache's next block.
+ * SDVG_STAGE: provisional write used once per denoise step so that attention
+ *   can read the block from the ring; the block it overwrites (block_index -
+ *   slots) is already outside the window of block_index.
+ * SDVG_FINAL: also records the block and advances next_block; *evicted_block
+ *   (host, may be NULL) receives the block that left the slot, -1 if it was empty
+ *   (always -1 for SDVG_STAGE).
+ * Errors: BAD_STATE (out of order), INVALID_ARG (flags), MISALIGNED.
+ */
+int sdvg_kv_commit(sdvg_cache* cache, const void* k_roped, const void* v,
+                   int64_t block_index, int flags, int64_t* evicted_block, void* stream);
+
+/*
+ * Fused step prologue: q_out = rope(q); rope(k) and v go straight into the ring
+ * slot of block_index with the semantics of `flags` above; k_out (optional)
+ * also receives rope(k) in the logical layout.  Bit-identical to
+ * sdvg_rope3d_qk followed by sdvg_kv_commit.  frame_offset is the first
+ * absolute latent frame of the block.  q/q_out may be NULL/NULL.
+ */
+int sdvg_rope3d_qk_commit(sdvg_cache* cache, const void* q, const void* k, const void* v,
+                          void* q_out, void* k_out,
+                          int frames, int grid_h, int grid_w, int frame_offset,
+                          const float* cos_sin_tab, int tab_frames,
+                          int64_t block_index, int flags, int64_t* evicted_block, void* stream);
+
+/* ---- block attention ---------------------------------------------------- */
+/*
+ * Device scratch needed by sdvg_block_attn_fwd (a few hundred bytes: a work
+ * counter and a status word).  256-byte aligned, caller-owned, must not be
+ * shared by calls that overlap on the device.
+ */
+size_t sdvg_block_attn_workspace_bytes(void);
+
+/*
+ * out[i, h, :] = sum_j softmax_j(scale * <q[i,h,:], K[j,h,:]>) V[j,h,:] where j
+ * runs over every token of the committed blocks visible to block_index (the
+ * last slots-1 blocks before it) and of block_index itself; no key is masked:
+ * bidirectional inside the block, causal across blocks (Sec. 4.1 "causal
+ * attention backbone with KV caching"; Sec. 1: blocks condition on earlier
+ * content through the shared cache).
+ *   q, out        device bf16 [block_tokens, heads, head_dim] of the cache's shape
+ *   k_self/v_self device bf16, same shape, the block's own roped K and V; both
+ *                 NULL means the block was staged (SDVG_STAGE) and is read from the ring
+ *   lse           optional device fp32 [heads, block_tokens]: log-sum-exp of the scaled logits
+ *   block_index   must be the cache's next block
+ * bf16 tensor-core products with fp32 accumulation, fp32 online softmax,
+ * probabilities rounded to bf16 before the second product.
+ * Errors: BAD_STATE (wrong block, self not staged), BAD_SHAPE, MISALIGNED,
+ * INVALID_ARG (workspace too small), UNSUPPORTED_ARCH, CUDA.
+ */
+int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self,
+                        const sdvg_cache* cache, int64_t block_index,
+                        void* out, float* lse, float scale,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronises `stream` and reports what the last attention launch that used
+ * `workspace` left in its status word: SDVG_OK, or SDVG_ERR_TIMEOUT if a
+ * bounded wait inside the kernel gave up (the output is then undefined).
+ */
+int sdvg_block_attn_status(const void* workspace, void* stream);
+
+/* ---- router ------------------------------------------------------------- */
+/*
+ * Eq. (1) and the policy of Sec. 3: q_min[b] = min_i scores[b, i];
+ * accept[b] = (first_block_index + b != 0) && (q_min[b] >= tau).
+ *   scores        device fp32, flat
+ *   frame_offsets device int32 [num_blocks+1] (block b owns scores[offsets[b]..offsets[b+1]))
+ *                 or NULL for frames_per_block consecutive scores per block
+ *   accept        device u8 [num_blocks]; q_min device fp32 [num_blocks];
+ *   argmin        optional device int32 [num_blocks]
+ * The minimum is the left-to-right strict-'<' minimum (ties and +0/-0 keep the
+ * lowest index); a NaN frame makes q_min that NaN and the block is rejected.
+ * With frame_offsets == NULL frames_per_block must be >= 1; with offsets every
+ * block must own at least one frame (checked on the device: a block with none
+ * gets accept 0, q_min NaN, argmin -1).
+ * Errors: INVALID_ARG, BAD_SHAPE (num_blocks < 0, frames_per_block < 1).
+ */
+int sdvg_route(const float* scores, const int32_t* frame_offsets,
+               int num_blocks, int frames_per_block, int64_t first_block_index, float tau,
+               uint8_t* accept, float* q_min, int32_t* argmin, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDVG_H_ */

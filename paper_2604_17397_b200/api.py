@@ -1,0 +1,252 @@
+"""Thin binding over the C ABI of libsdvg (see include/sdvg.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch supplies device memory and the current stream.  There is no
+fallback: if the shared library is missing or a call fails, an exception is
+raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsdvg.so")
+
+SDVG_OK = 0
+SDVG_ERR_INVALID_ARG = 1
+SDVG_ERR_BAD_SHAPE = 2
+SDVG_ERR_MISALIGNED = 3
+SDVG_ERR_BAD_STATE = 4
+SDVG_ERR_UNSUPPORTED_ARCH = 5
+SDVG_ERR_CUDA = 6
+SDVG_ERR_TIMEOUT = 7
+SDVG_STAGE = 1
+SDVG_FINAL = 2
+
+# name -> (restype, argtypes); the list of everything include/sdvg.h declares
+_VP, _I, _I64, _SZ, _F = C.c_void_p, C.c_int, C.c_int64, C.c_size_t, C.c_float
+SIGNATURES = {
+    "sdvg_status_string": (C.c_char_p, [_I]),
+    "sdvg_last_cuda_error": (_I, []),
+    "sdvg_last_cuda_error_string": (C.c_char_p, []),
+    "sdvg_rope3d_pairs": (_I, [_I, C.POINTER(_I), C.POINTER(_I), C.POINTER(_I)]),
+    "sdvg_rope3d_table_floats": (_SZ, [_I, _I, _I, _I]),
+    "sdvg_rope3d_table": (_I, [_VP, _I, _I, _I, _I]),
+    "sdvg_rope3d_qk": (_I, [_VP, _VP, _VP, _VP, _I, _I, _I, _I, _I, _I, _I, _VP, _I, _VP]),
+    "sdvg_cache_bytes": (_SZ, [_I, _I, _I, _I]),
+    "sdvg_cache_create": (_I, [C.POINTER(_VP), _VP, _VP, _I, _I, _I, _I]),
+    "sdvg_cache_reset": (_I, [_VP]),
+    "sdvg_cache_destroy": (_I, [_VP]),
+    "sdvg_cache_state": (_I, [_VP, C.POINTER(_I64), C.POINTER(_I64), C.POINTER(_I64)]),
+    "sdvg_cache_read_block": (_I, [_VP, _I, _VP, _VP, _VP]),
+    "sdvg_kv_commit": (_I, [_VP, _VP, _VP, _I64, _I, C.POINTER(_I64), _VP]),
+    "sdvg_rope3d_qk_commit": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
+                                   C.POINTER(_I64), _VP]),
+    "sdvg_block_attn_workspace_bytes": (_SZ, []),
+    "sdvg_block_attn_fwd": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
+    "sdvg_block_attn_status": (_I, [_VP, _VP]),
+    "sdvg_route": (_I, [_VP, _VP, _I, _I, _I64, _F, _VP, _VP, _VP, _VP]),
+}
+
+_lib = None
+
+
+class SdvgError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().sdvg_status_string(status).decode()
+        if status == SDVG_ERR_CUDA:
+            msg += ": " + lib().sdvg_last_cuda_error_string().decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def lib() -> C.CDLL:
+    """Load libsdvg.so (built in-tree by ``build.py``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: run `python -m paper_2604_17397_b200.build` first")
+        l = C.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != SDVG_OK:
+        raise SdvgError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _bf16(t: Optional[torch.Tensor], shape=None):
+    if t is None:
+        return None
+    if t.dtype != torch.bfloat16:
+        raise ValueError("expected a bfloat16 tensor")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return _ptr(t)
+
+
+# ---------------------------------------------------------------- RoPE
+
+def sdvg_rope3d_pairs(head_dim: int):
+    pf, ph, pw = _I(), _I(), _I()
+    _check(lib().sdvg_rope3d_pairs(head_dim, C.byref(pf), C.byref(ph), C.byref(pw)), "sdvg_rope3d_pairs")
+    return pf.value, ph.value, pw.value
+
+
+def sdvg_rope3d_table(head_dim: int, tab_frames: int, grid_h: int, grid_w: int) -> torch.Tensor:
+    """Host fp32 (cos, sin) table built by the library; upload it with ``.cuda()``."""
+    n = lib().sdvg_rope3d_table_floats(head_dim, tab_frames, grid_h, grid_w)
+    if n == 0:
+        raise SdvgError(SDVG_ERR_BAD_SHAPE, "sdvg_rope3d_table_floats")
+    out = torch.empty(n, dtype=torch.float32)
+    _check(lib().sdvg_rope3d_table(out.data_ptr(), head_dim, tab_frames, grid_h, grid_w), "sdvg_rope3d_table")
+    return out
+
+
+def sdvg_rope3d_qk(q, k, q_out, k_out, grid, frame_offset: int, table: torch.Tensor, tab_frames: int,
+                   stream=None) -> None:
+    ref = q if q is not None else k
+    tokens, heads, head_dim = ref.shape
+    frames, grid_h, grid_w = grid
+    st = lib().sdvg_rope3d_qk(_bf16(q), _bf16(k), _bf16(q_out, None if q is None else q.shape),
+                              _bf16(k_out, None if k is None else k.shape), tokens, heads, head_dim,
+                              frames, grid_h, grid_w, frame_offset, _ptr(table), tab_frames, _stream(stream))
+    _check(st, "sdvg_rope3d_qk")
+
+
+# ---------------------------------------------------------------- cache
+
+class Cache:
+    """Rolling KV cache: torch owns the two device buffers, the library the ring state."""
+
+    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int, device="cuda"):
+        nbytes = lib().sdvg_cache_bytes(slots, heads, block_tokens, head_dim)
+        if nbytes == 0:
+            raise SdvgError(SDVG_ERR_BAD_SHAPE, "sdvg_cache_bytes")
+        self.slots, self.heads, self.block_tokens, self.head_dim = slots, heads, block_tokens, head_dim
+        # physical layout [heads][slots][tokens][dim]; torch's allocator aligns to 512 B, so over-allocate
+        self._k_raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+        self._v_raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+        self.k_ptr = (self._k_raw.data_ptr() + 1023) & ~1023
+        self.v_ptr = (self._v_raw.data_ptr() + 1023) & ~1023
+        h = _VP()
+        _check(lib().sdvg_cache_create(C.byref(h), self.k_ptr, self.v_ptr, slots, heads, block_tokens, head_dim),
+               "sdvg_cache_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle.value:
+            lib().sdvg_cache_destroy(self.handle)
+            self.handle = _VP()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self):
+        _check(lib().sdvg_cache_reset(self.handle), "sdvg_cache_reset")
+
+    def state(self):
+        """(next_block, [slot -> committed block or -1], staged_block)."""
+        nb, sb = _I64(), _I64()
+        arr = (_I64 * self.slots)()
+        _check(lib().sdvg_cache_state(self.handle, C.byref(nb), arr, C.byref(sb)), "sdvg_cache_state")
+        return nb.value, list(arr), sb.value
+
+    def read_block(self, slot: int, stream=None):
+        """Logical [tokens, heads, dim] copies of the K and V held in ``slot``."""
+        shape = (self.block_tokens, self.heads, self.head_dim)
+        k = torch.empty(shape, dtype=torch.bfloat16, device=self._k_raw.device)
+        v = torch.empty_like(k)
+        _check(lib().sdvg_cache_read_block(self.handle, slot, k.data_ptr(), v.data_ptr(), _stream(stream)),
+               "sdvg_cache_read_block")
+        return k, v
+
+
+def sdvg_kv_commit(cache: Cache, k_roped, v, block_index: int, flags: int, stream=None) -> int:
+    """Returns the evicted block (-1 if none)."""
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    ev = _I64(-1)
+    st = lib().sdvg_kv_commit(cache.handle, _bf16(k_roped, shape), _bf16(v, shape), block_index, flags,
+                              C.byref(ev), _stream(stream))
+    _check(st, "sdvg_kv_commit")
+    return ev.value
+
+
+def sdvg_rope3d_qk_commit(cache: Cache, q, k, v, q_out, k_out, grid, frame_offset: int, table, tab_frames: int,
+                          block_index: int, flags: int, stream=None) -> int:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    frames, grid_h, grid_w = grid
+    ev = _I64(-1)
+    st = lib().sdvg_rope3d_qk_commit(cache.handle, _bf16(q, None if q is None else shape), _bf16(k, shape),
+                                     _bf16(v, shape), _bf16(q_out, None if q_out is None else shape),
+                                     _bf16(k_out, None if k_out is None else shape),
+                                     frames, grid_h, grid_w, frame_offset, _ptr(table), tab_frames,
+                                     block_index, flags, C.byref(ev), _stream(stream))
+    _check(st, "sdvg_rope3d_qk_commit")
+    return ev.value
+
+
+# ---------------------------------------------------------------- attention
+
+def attn_workspace(device="cuda", extra_bytes: int = 0) -> torch.Tensor:
+    n = lib().sdvg_block_attn_workspace_bytes() + extra_bytes
+    raw = torch.zeros(n + 256, dtype=torch.uint8, device=device)
+    off = (-raw.data_ptr()) % 256
+    return raw[off:off + n]
+
+
+def sdvg_block_attn_fwd(q, k_self, v_self, cache: Cache, block_index: int, out, lse, scale: float,
+                        workspace: torch.Tensor, stream=None) -> None:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    if lse is not None and (lse.dtype != torch.float32 or tuple(lse.shape) != (cache.heads, cache.block_tokens)):
+        raise ValueError("lse must be float32 [heads, block_tokens]")
+    st = lib().sdvg_block_attn_fwd(_bf16(q, shape), _bf16(k_self, None if k_self is None else shape),
+                                   _bf16(v_self, None if v_self is None else shape), cache.handle, block_index,
+                                   _bf16(out, shape), _ptr(lse), scale, workspace.data_ptr(), workspace.numel(),
+                                   _stream(stream))
+    _check(st, "sdvg_block_attn_fwd")
+
+
+def sdvg_block_attn_status(workspace: torch.Tensor, stream=None) -> int:
+    return lib().sdvg_block_attn_status(workspace.data_ptr(), _stream(stream))
+
+
+# ---------------------------------------------------------------- router
+
+def sdvg_route(scores, frame_offsets, num_blocks: int, frames_per_block: int, first_block_index: int, tau: float,
+               accept, q_min, argmin=None, stream=None) -> None:
+    if scores.dtype != torch.float32 or q_min.dtype != torch.float32 or accept.dtype != torch.uint8:
+        raise ValueError("scores/q_min must be float32 and accept uint8")
+    if frame_offsets is not None and frame_offsets.dtype != torch.int32:
+        raise ValueError("frame_offsets must be int32")
+    if argmin is not None and argmin.dtype != torch.int32:
+        raise ValueError("argmin must be int32")
+    st = lib().sdvg_route(_ptr(scores), _ptr(frame_offsets), num_blocks, frames_per_block, first_block_index, tau,
+                          _ptr(accept), _ptr(q_min), _ptr(argmin), _stream(stream))
+    _check(st, "sdvg_route")

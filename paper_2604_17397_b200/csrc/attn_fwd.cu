@@ -1,0 +1,420 @@
+// Block attention forward for sm_100a: O = softmax(scale * Q K^T) V over every visible key
+// (Sec. 4.1: causal attention backbone with KV caching; no key is masked inside a call because the
+// block sees all of itself and all of its window).
+//
+// Both products run on the 5th-generation tensor cores (tcgen05.mma, bf16 in, fp32 accumulators in
+// tensor memory).  Q, K and V tiles are staged in shared memory by TMA with the 128-byte swizzle;
+// S = Q K^T lands in TMEM, the softmax threads (one per query row) read it with tcgen05.ld, write
+// the bf16 probabilities back over the same TMEM columns, and O += P V takes P straight from TMEM
+// and V from shared memory as an MN-major operand.  Keys arrive as up to three segments (runs of
+// ring slots and/or the block's own K/V tensors), each with its own tensor map whose row extent
+// ends at the segment so that TMA zero-fills the ragged last tile; those columns are masked to
+// -inf before the row maximum.
+//
+// Every wait on an mbarrier is bounded: after kWaitLimitNs the waiting thread raises an abort flag
+// and writes SDVG_ERR_TIMEOUT to the status word; all roles then fall through to the common exit,
+// which releases tensor memory.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "sdvg_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kTileM = 128;            // query rows per tile
+constexpr int kTileN = 128;            // keys per tile
+constexpr int kMaxSegments = 3;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr int kWorkspaceBytes = 256;
+
+struct alignas(64) AttnParams {
+  CUtensorMap q_map;
+  CUtensorMap k_map[kMaxSegments];
+  CUtensorMap v_map[kMaxSegments];
+  int seg_len[kMaxSegments];
+  int nseg;
+  int tokens, heads;
+  float scale_log2e;                   // scale * log2(e): softmax is evaluated with exp2
+  __nv_bfloat16* out;
+  float* lse;
+  unsigned int* work;                  // [0] work counter, [1] status word
+#ifdef SDVG_ATTN_DEBUG
+  float* dbg;                          // S, P, O of the first key tile of CTA (0, 0)
+#endif
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct WaitCtx {
+  volatile int* abort_flag;            // shared
+  unsigned int* status;                // global
+  uint64_t t0;
+};
+
+// Bounded mbarrier wait.  Returns false once the CTA is aborting.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, const WaitCtx& c) {
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0xff) == 0xff) {
+      if (*c.abort_flag) return false;
+      if (globaltimer_ns() - c.t0 > kWaitLimitNs) {
+        *c.abort_flag = 1;
+        atomicExch(c.status, (unsigned)SDVG_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+template <int D>
+struct SimpleSmem {
+  static constexpr int kHalves = D / 64;                 // 64-column (128-byte) swizzle panels
+  static constexpr int kPanelBytes = kTileN * 128;       // 128 rows x 128 B
+  static constexpr int kTileBytes = kHalves * kPanelBytes;
+  static constexpr int kQ = 0;
+  static constexpr int kK = kTileBytes;
+  static constexpr int kV = 2 * kTileBytes;
+  static constexpr int kBars = 3 * kTileBytes;
+  static constexpr int kTotal = kBars + 64;
+  static constexpr int kDynamic = kTotal + 1024;         // slack for the 1024-byte alignment
+};
+
+// One CTA = one 128-row query tile of one head, four warps, no overlap between the stages.
+template <int D>
+__global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_constant__ AttnParams p) {
+  using L = SimpleSmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::kBars);
+  uint64_t* s_bar = full_bar + 1;
+  uint64_t* o_bar = full_bar + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 3);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int qt = blockIdx.x, head = blockIdx.y;
+  constexpr uint32_t kTmemCols = 256;                    // S: [0,128) (P aliases its first 64), O: [128, 128+D)
+
+  if (tid == 0) {
+    mbar_init(full_bar, 1);
+    mbar_init(s_bar, 1);
+    mbar_init(o_bar, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&p.q_map);
+  }
+  if (warp == 0) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tS = tmem_base, tO = tmem_base + 128;
+  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  WaitCtx wc{abort_flag, p.work + 1, globaltimer_ns()};
+
+  uint32_t full_phase = 0, s_phase = 0, o_phase = 0;
+  bool alive = true;
+
+  if (tid == 0) {
+    mbar_expect_tx(full_bar, L::kTileBytes);
+    for (int h = 0; h < L::kHalves; ++h)
+      tma_load_3d(smem + L::kQ + h * L::kPanelBytes, &p.q_map, full_bar, h * 64, qt * kTileM, head);
+  }
+  alive = wait_bar(full_bar, full_phase, wc);
+  full_phase ^= 1;
+
+  constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, false);
+  constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, true);
+  const uint32_t sQ = smem_u32(smem + L::kQ), sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
+
+  float m_run = -INFINITY, l_run = 0.f;
+  int it = 0;
+  for (int seg = 0; seg < p.nseg && alive; ++seg) {
+    const int len = p.seg_len[seg];
+    const int ntiles = (len + kTileN - 1) / kTileN;
+    for (int kt = 0; kt < ntiles && alive; ++kt, ++it) {
+      const int valid = min(kTileN, len - kt * kTileN);
+      if (tid == 0) {
+        mbar_expect_tx(full_bar, 2 * L::kTileBytes);
+        for (int h = 0; h < L::kHalves; ++h) {
+          tma_load_3d(smem + L::kK + h * L::kPanelBytes, &p.k_map[seg], full_bar, h * 64, kt * kTileN, head);
+          tma_load_3d(smem + L::kV + h * L::kPanelBytes, &p.v_map[seg], full_bar, h * 64, kt * kTileN, head);
+        }
+      }
+      if (!(alive = wait_bar(full_bar, full_phase, wc))) break;
+      full_phase ^= 1;
+      if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * L::kPanelBytes + (kk & 3) * 32;   // 16 bf16 = 32 B along K
+          mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), kIdescQK,
+                 kk > 0);
+        }
+        mma_commit(s_bar);
+      }
+      if (!(alive = wait_bar(s_bar, s_phase, wc))) break;
+      s_phase ^= 1;
+      tc_fence_after();
+
+      // ---- softmax of this thread's row ---------------------------------------------------
+      uint32_t s[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, s[c]);
+      tmem_wait_ld();
+#ifdef SDVG_ATTN_DEBUG
+      if (p.dbg && qt == 0 && head == 0 && it == 0)
+        for (int c = 0; c < 4; ++c)
+          for (int j = 0; j < 32; ++j) p.dbg[tid * 128 + c * 32 + j] = __uint_as_float(s[c][j]);
+#endif
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float x = __uint_as_float(s[c][j]) * p.scale_log2e;
+          if (c * 32 + j >= valid) x = -INFINITY;
+          s[c][j] = __float_as_uint(x);
+          mx = fmaxf(mx, x);
+        }
+      const float m_new = fmaxf(m_run, mx);
+      const float alpha = fast_exp2(m_run - m_new);
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float p0 = fast_exp2(__uint_as_float(s[c][2 * j]) - m_new);
+          const float p1 = fast_exp2(__uint_as_float(s[c][2 * j + 1]) - m_new);
+          sum += p0 + p1;
+          __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+          pk[j] = *reinterpret_cast<uint32_t*>(&b);
+        }
+        tmem_st16(tS + lane_off + c * 16, pk);     // P overwrites S columns already held in registers
+      }
+      l_run = l_run * alpha + sum;
+      m_run = m_new;
+      if (it > 0) {
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tO + lane_off + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+          tmem_st32(tO + lane_off + c * 32, o);
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      __syncthreads();
+      if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kTileN / 16; ++kk) {
+          // 16 keys = two 8-row groups of the V panel; the two 64-column panels are kPanelBytes apart
+          mma_ts(tO, tS + kk * 8, smem_desc_sw128(sV + kk * 2048, L::kPanelBytes, 1024), kIdescPV,
+                 (it > 0 || kk > 0) ? 1u : 0u);
+        }
+        mma_commit(o_bar);
+      }
+      if (!(alive = wait_bar(o_bar, o_phase, wc))) break;
+      o_phase ^= 1;
+      tc_fence_after();
+#ifdef SDVG_ATTN_DEBUG
+      if (p.dbg && qt == 0 && head == 0 && it == 0) {
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tS + lane_off + c * 32, r);
+          tmem_wait_ld();
+          for (int j = 0; j < 32; ++j) p.dbg[128 * 128 + tid * 64 + c * 32 + j] = __uint_as_float(r[j]);
+        }
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tO + lane_off + c * 32, r);
+          tmem_wait_ld();
+          for (int j = 0; j < 32; ++j) p.dbg[128 * 128 + 128 * 64 + tid * D + c * 32 + j] = __uint_as_float(r[j]);
+        }
+      }
+#endif
+    }
+  }
+
+  // ---- epilogue: O / l -> bf16, this thread's row ------------------------------------------
+  const int row = qt * kTileM + tid;
+  if (alive && it > 0) {
+    const float inv = 1.f / l_run;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t o[32];
+      tmem_ld32(tO + lane_off + c * 32, o);
+      tmem_wait_ld();
+      if (row < p.tokens) {
+        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)row * p.heads + head) * D + c * 32);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * e]) * inv,
+                                                     __uint_as_float(o[v * 8 + 2 * e + 1]) * inv);
+            w[e] = *reinterpret_cast<uint32_t*>(&b);
+          }
+          dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+    if (p.lse && row < p.tokens)
+      p.lse[(size_t)head * p.tokens + row] = m_run * 0.6931471805599453f + logf(l_run);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ---- host side -------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 matrix seen as (dim, rows, heads) with arbitrary row and head strides; box = 64 x 128 x 1,
+// 128-byte swizzle, rows beyond `rows` read as zero.
+int make_map(CUtensorMap* m, const void* base, int head_dim, long long rows, int heads, size_t row_stride_bytes,
+             size_t head_stride_bytes) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return SDVG_ERR_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)rows, (cuuint64_t)heads};
+  cuuint64_t strides[2] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)head_stride_bytes};
+  cuuint32_t box[3] = {64, (cuuint32_t)kTileN, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SDVG_OK : SDVG_ERR_CUDA;
+}
+
+template <int D>
+int launch_simple(const AttnParams& p, cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_simple_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SimpleSmem<D>::kDynamic);
+    if (e != cudaSuccess) return sdvg::cuda_status(e);
+    configured = true;
+  }
+  dim3 grid((p.tokens + kTileM - 1) / kTileM, p.heads);
+  attn_fwd_simple_kernel<D><<<grid, 128, SimpleSmem<D>::kDynamic, stream>>>(p);
+  return sdvg::cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t sdvg_block_attn_workspace_bytes(void) { return kWorkspaceBytes; }
+
+int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
+                        int64_t block_index, void* out, float* lse, float scale, void* workspace,
+                        size_t workspace_bytes, void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!q || !c || !out || !workspace) return SDVG_ERR_INVALID_ARG;
+  if ((k_self == nullptr) != (v_self == nullptr)) return SDVG_ERR_INVALID_ARG;
+  if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
+  if (!(scale > 0.f) || !isfinite(scale)) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(q) || !sdvg::aligned16(k_self) || !sdvg::aligned16(v_self) || !sdvg::aligned16(out) ||
+      (reinterpret_cast<uintptr_t>(lse) & 3) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return SDVG_ERR_MISALIGNED;
+  if (block_index < 0 || block_index != c->next_block) return SDVG_ERR_BAD_STATE;
+  if (!k_self && c->staged_block != block_index) return SDVG_ERR_BAD_STATE;
+  int st = sdvg::require_sm100();
+  if (st != SDVG_OK) return st;
+
+  const int T = c->block_tokens, H = c->heads, D = c->head_dim, S = c->slots;
+  const size_t row_bytes = (size_t)D * 2;
+  const size_t ring_head_stride = (size_t)S * T * row_bytes;
+  AttnParams p = {};
+  p.tokens = T;
+  p.heads = H;
+  p.scale_log2e = scale * 1.4426950408889634f;
+  p.out = (__nv_bfloat16*)out;
+  p.lse = lse;
+  p.work = (unsigned int*)workspace;
+  if ((st = make_map(&p.q_map, q, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+
+  // Visible committed blocks: the last S-1 before block_index, living in slots (b % S).  Their slots
+  // form at most two runs of consecutive slots; with the block staged, its slot joins them.
+  const int64_t first = block_index - (S - 1) > 0 ? block_index - (S - 1) : 0;
+  bool use[64];
+  if (S > 64) return SDVG_ERR_BAD_SHAPE;
+  for (int s = 0; s < S; ++s) use[s] = false;
+  for (int64_t b = first; b < block_index; ++b) {
+    const int s = (int)(b % S);
+    if (c->slot_block[s] != b) return SDVG_ERR_BAD_STATE;
+    use[s] = true;
+  }
+  if (!k_self) use[(int)(block_index % S)] = true;
+  for (int s = 0; s < S;) {
+    if (!use[s]) { ++s; continue; }
+    int e = s;
+    while (e < S && use[e]) ++e;
+    if (p.nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
+    const long long rows = (long long)(e - s) * T;
+    const char* kb = (const char*)c->k_buf + (size_t)s * T * row_bytes;
+    const char* vb = (const char*)c->v_buf + (size_t)s * T * row_bytes;
+    if ((st = make_map(&p.k_map[p.nseg], kb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
+    if ((st = make_map(&p.v_map[p.nseg], vb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
+    p.seg_len[p.nseg++] = (int)rows;
+    s = e;
+  }
+  if (k_self) {
+    if (p.nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
+    if ((st = make_map(&p.k_map[p.nseg], k_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+    if ((st = make_map(&p.v_map[p.nseg], v_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+    p.seg_len[p.nseg++] = T;
+  }
+#ifdef SDVG_ATTN_DEBUG
+  p.dbg = workspace_bytes >= (size_t)kWorkspaceBytes + 4 * (128 * 128 + 128 * 64 + 128 * 128)
+              ? (float*)((char*)workspace + kWorkspaceBytes)
+              : nullptr;
+#endif
+  cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  return D == 128 ? launch_simple<128>(p, stream) : launch_simple<64>(p, stream);
+}
+
+int sdvg_block_attn_status(const void* workspace, void* stream_) {
+  if (!workspace) return SDVG_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  unsigned int w[2] = {0, 0};
+  cudaError_t e = cudaMemcpyAsync(w, workspace, sizeof(w), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  return w[1] == 0 ? SDVG_OK : (int)w[1];
+}
+
+}  // extern "C"

@@ -1,0 +1,264 @@
+// 3D-RoPE, ring commit and their fusion: one streaming pass over HBM per tensor.
+//
+// Every thread owns one 16-byte column slice (8 bf16 = 4 rotary pairs) of one token and walks a
+// group of heads with it, so the token's (frame, row, column) split and its (cos, sin) pairs are
+// fetched once and reused for every head; loads of a head group are issued before the first use
+// so that several 16-byte requests per thread are in flight.  Reads use the logical
+// [tokens, heads, dim] layout; writes go to the logical layout and/or to the ring slot
+// ([heads][slots][tokens][dim]).  Both sides move whole 16-byte vectors, 128/256 contiguous
+// bytes per (token, head) row.
+#include <cuda_bf16.h>
+
+#include "sdvg_internal.h"
+
+namespace {
+
+constexpr int kMaxJobs = 3;
+constexpr int kHeadGroup = 8;     // heads walked by one thread
+constexpr int kThreads = 256;
+
+struct TensorJob {
+  const uint4* src;        // [tokens, heads, dim] bf16
+  uint4* dst_logical;      // same layout, or nullptr
+  uint4* dst_slot;         // points at (head 0, slot, token 0): head stride = slots*tokens*dim, or nullptr
+  int rope;                // rotate pairs (q, k) or copy (v)
+};
+
+struct RopeCommitParams {
+  TensorJob job[kMaxJobs];
+  int njobs;
+  int tokens, heads;
+  int grid_hw, grid_w;     // grid_h*grid_w and grid_w of the latent grid
+  int frame_offset;
+  int pairs_f, pairs_h;    // pair split: [0,pf) frame, [pf,pf+ph) row, rest column
+  int tab_h_off, tab_w_off;  // float offsets of the row and column sub-tables
+  long long slot_head_stride_vec;  // 16-byte vectors between consecutive heads in the ring buffer
+  const float2* tab;
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// One pair: re' = fl(fl(re*c) - fl(im*s)), im' = fl(fl(re*s) + fl(im*c)); RNE pack to bf16x2.
+__device__ __forceinline__ uint32_t rotate_pair(uint32_t w, float2 cs) {
+  float re = bf16_lo(w), im = bf16_hi(w);
+  float r0 = __fsub_rn(__fmul_rn(re, cs.x), __fmul_rn(im, cs.y));
+  float r1 = __fadd_rn(__fmul_rn(re, cs.y), __fmul_rn(im, cs.x));
+  __nv_bfloat162 p = __floats2bfloat162_rn(r0, r1);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads) rope_commit_kernel(const __grid_constant__ RopeCommitParams p) {
+  constexpr int VPR = D / 8;                       // 16-byte vectors per (token, head) row
+  const TensorJob job = p.job[blockIdx.z];
+  const int h0 = blockIdx.y * kHeadGroup;
+  const int nh = min(kHeadGroup, p.heads - h0);
+  const int total = p.tokens * VPR;
+  for (int i = blockIdx.x * kThreads + threadIdx.x; i < total; i += gridDim.x * kThreads) {
+    const int t = i / VPR;
+    const int j = i - t * VPR;
+    float2 cs[4];
+    if (job.rope) {
+      const int f = t / p.grid_hw;
+      const int rem = t - f * p.grid_hw;
+      const int y = rem / p.grid_w;
+      const int x = rem - y * p.grid_w;
+      const int pairs_w = D / 2 - p.pairs_f - p.pairs_h;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int pr = 4 * j + e;
+        int idx;
+        if (pr < p.pairs_f) idx = (p.frame_offset + f) * p.pairs_f + pr;
+        else if (pr < p.pairs_f + p.pairs_h) idx = p.tab_h_off + y * p.pairs_h + (pr - p.pairs_f);
+        else idx = p.tab_w_off + x * pairs_w + (pr - p.pairs_f - p.pairs_h);
+        cs[e] = __ldg(p.tab + idx);
+      }
+    }
+    const size_t row0 = ((size_t)t * p.heads + h0) * VPR + j;     // vector index of (t, h0, j)
+    uint4 v[kHeadGroup];
+#pragma unroll
+    for (int g = 0; g < kHeadGroup; ++g)
+      if (g < nh) v[g] = __ldcs(job.src + row0 + (size_t)g * VPR);
+#pragma unroll
+    for (int g = 0; g < kHeadGroup; ++g) {
+      if (g < nh) {
+        uint4 w = v[g];
+        if (job.rope) {
+          w.x = rotate_pair(w.x, cs[0]);
+          w.y = rotate_pair(w.y, cs[1]);
+          w.z = rotate_pair(w.z, cs[2]);
+          w.w = rotate_pair(w.w, cs[3]);
+        }
+        if (job.dst_logical) __stcs(job.dst_logical + row0 + (size_t)g * VPR, w);
+        if (job.dst_slot)
+          job.dst_slot[(size_t)(h0 + g) * p.slot_head_stride_vec + (size_t)t * VPR + j] = w;
+      }
+    }
+  }
+}
+
+// Ring slot -> logical layout (accessor used to inspect the cache).
+template <int D>
+__global__ void __launch_bounds__(kThreads) slot_read_kernel(const uint4* __restrict__ slot_base,
+                                                              uint4* __restrict__ dst, int tokens, int heads,
+                                                              long long slot_head_stride_vec) {
+  constexpr int VPR = D / 8;
+  const long long total = (long long)tokens * heads * VPR;
+  for (long long i = (long long)blockIdx.x * kThreads + threadIdx.x; i < total;
+       i += (long long)gridDim.x * kThreads) {
+    const int j = (int)(i % VPR);
+    const long long row = i / VPR;
+    const int h = (int)(row % heads);
+    const long long t = row / heads;
+    dst[i] = slot_base[(long long)h * slot_head_stride_vec + t * VPR + j];
+  }
+}
+
+struct RopeArgs {
+  int frames, grid_h, grid_w, frame_offset, tab_frames;
+  const float* tab;
+};
+
+int fill_rope(RopeCommitParams& p, int head_dim, int tokens, const RopeArgs& r) {
+  if (r.frames <= 0 || r.grid_h <= 0 || r.grid_w <= 0) return SDVG_ERR_BAD_SHAPE;
+  if ((long long)r.frames * r.grid_h * r.grid_w != tokens) return SDVG_ERR_BAD_SHAPE;
+  if (!r.tab) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(r.tab)) return SDVG_ERR_MISALIGNED;
+  if (r.tab_frames <= 0) return SDVG_ERR_BAD_SHAPE;
+  if (r.frame_offset < 0 || (long long)r.frame_offset + r.frames > r.tab_frames) return SDVG_ERR_BAD_STATE;
+  int pf, ph, pw;
+  sdvg_rope3d_pairs(head_dim, &pf, &ph, &pw);
+  p.grid_hw = r.grid_h * r.grid_w;
+  p.grid_w = r.grid_w;
+  p.frame_offset = r.frame_offset;
+  p.pairs_f = pf;
+  p.pairs_h = ph;
+  p.tab_h_off = r.tab_frames * pf;                 // in (cos, sin) pairs
+  p.tab_w_off = p.tab_h_off + r.grid_h * ph;
+  p.tab = reinterpret_cast<const float2*>(r.tab);
+  return SDVG_OK;
+}
+
+int launch(RopeCommitParams& p, int head_dim, cudaStream_t stream) {
+  if (p.njobs == 0) return SDVG_OK;
+  const int vpr = head_dim / 8;
+  const long long total = (long long)p.tokens * vpr;
+  if (total * p.heads >= (1ll << 31)) return SDVG_ERR_BAD_SHAPE;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int groups = (p.heads + kHeadGroup - 1) / kHeadGroup;
+  long long want = (total + kThreads - 1) / kThreads;
+  // a whole number of waves: up to 8 resident 256-thread blocks per SM shared by the (y, z) slices
+  long long cap = (long long)sms * 8 / (groups * p.njobs);
+  if (cap < 1) cap = 1;
+  dim3 grid((unsigned)(want < cap ? want : cap), groups, p.njobs);
+  if (head_dim == 128) rope_commit_kernel<128><<<grid, kThreads, 0, stream>>>(p);
+  else rope_commit_kernel<64><<<grid, kThreads, 0, stream>>>(p);
+  return sdvg::cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+extern "C" {
+
+int sdvg_rope3d_qk(const void* q, const void* k, void* q_out, void* k_out, int tokens, int heads,
+                   int head_dim, int frames, int grid_h, int grid_w, int frame_offset,
+                   const float* cos_sin_tab, int tab_frames, void* stream) {
+  if ((q == nullptr) != (q_out == nullptr) || (k == nullptr) != (k_out == nullptr)) return SDVG_ERR_INVALID_ARG;
+  if (!q && !k) return SDVG_ERR_INVALID_ARG;
+  if (tokens <= 0 || heads <= 0 || !sdvg::head_dim_ok(head_dim)) return SDVG_ERR_BAD_SHAPE;
+  if (!sdvg::aligned16(q) || !sdvg::aligned16(k) || !sdvg::aligned16(q_out) || !sdvg::aligned16(k_out))
+    return SDVG_ERR_MISALIGNED;
+  RopeCommitParams p = {};
+  p.tokens = tokens;
+  p.heads = heads;
+  int st = fill_rope(p, head_dim, tokens, RopeArgs{frames, grid_h, grid_w, frame_offset, tab_frames, cos_sin_tab});
+  if (st != SDVG_OK) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  if (q) p.job[p.njobs++] = TensorJob{(const uint4*)q, (uint4*)q_out, nullptr, 1};
+  if (k) p.job[p.njobs++] = TensorJob{(const uint4*)k, (uint4*)k_out, nullptr, 1};
+  return launch(p, head_dim, (cudaStream_t)stream);
+}
+
+int sdvg_kv_commit(sdvg_cache* c, const void* k_roped, const void* v, int64_t block_index, int flags,
+                   int64_t* evicted_block, void* stream) {
+  if (!c || !k_roped || !v) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(k_roped) || !sdvg::aligned16(v)) return SDVG_ERR_MISALIGNED;
+  int slot = 0;
+  int st = sdvg::ring_begin_commit(c, block_index, flags, &slot);
+  if (st != SDVG_OK) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  RopeCommitParams p = {};
+  p.tokens = c->block_tokens;
+  p.heads = c->heads;
+  p.slot_head_stride_vec = (long long)c->slots * c->block_tokens * (c->head_dim / 8);
+  uint4* kslot = (uint4*)c->k_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  uint4* vslot = (uint4*)c->v_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  p.job[p.njobs++] = TensorJob{(const uint4*)k_roped, nullptr, kslot, 0};
+  p.job[p.njobs++] = TensorJob{(const uint4*)v, nullptr, vslot, 0};
+  st = launch(p, c->head_dim, (cudaStream_t)stream);
+  if (st != SDVG_OK) return st;
+  sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
+  return SDVG_OK;
+}
+
+int sdvg_rope3d_qk_commit(sdvg_cache* c, const void* q, const void* k, const void* v, void* q_out,
+                          void* k_out, int frames, int grid_h, int grid_w, int frame_offset,
+                          const float* cos_sin_tab, int tab_frames, int64_t block_index, int flags,
+                          int64_t* evicted_block, void* stream) {
+  if (!c || !k || !v) return SDVG_ERR_INVALID_ARG;
+  if ((q == nullptr) != (q_out == nullptr)) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(q) || !sdvg::aligned16(k) || !sdvg::aligned16(v) || !sdvg::aligned16(q_out) ||
+      !sdvg::aligned16(k_out))
+    return SDVG_ERR_MISALIGNED;
+  RopeCommitParams p = {};
+  p.tokens = c->block_tokens;
+  p.heads = c->heads;
+  int st = fill_rope(p, c->head_dim, c->block_tokens,
+                     RopeArgs{frames, grid_h, grid_w, frame_offset, tab_frames, cos_sin_tab});
+  if (st != SDVG_OK) return st;
+  int slot = 0;
+  if ((st = sdvg::ring_begin_commit(c, block_index, flags, &slot)) != SDVG_OK) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  p.slot_head_stride_vec = (long long)c->slots * c->block_tokens * (c->head_dim / 8);
+  uint4* kslot = (uint4*)c->k_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  uint4* vslot = (uint4*)c->v_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  if (q) p.job[p.njobs++] = TensorJob{(const uint4*)q, (uint4*)q_out, nullptr, 1};
+  p.job[p.njobs++] = TensorJob{(const uint4*)k, (uint4*)k_out, kslot, 1};
+  p.job[p.njobs++] = TensorJob{(const uint4*)v, nullptr, vslot, 0};
+  st = launch(p, c->head_dim, (cudaStream_t)stream);
+  if (st != SDVG_OK) return st;
+  sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
+  return SDVG_OK;
+}
+
+int sdvg_cache_read_block(const sdvg_cache* c, int slot, void* k_out, void* v_out, void* stream) {
+  if (!c || (!k_out && !v_out)) return SDVG_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= c->slots) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(k_out) || !sdvg::aligned16(v_out)) return SDVG_ERR_MISALIGNED;
+  int st = sdvg::require_sm100();
+  if (st != SDVG_OK) return st;
+  const long long stride = (long long)c->slots * c->block_tokens * (c->head_dim / 8);
+  const long long total = (long long)c->block_tokens * c->heads * (c->head_dim / 8);
+  const unsigned blocks = (unsigned)((total + kThreads - 1) / kThreads < 148 * 8 ? (total + kThreads - 1) / kThreads
+                                                                                  : 148 * 8);
+  const void* bufs[2] = {c->k_buf, c->v_buf};
+  void* outs[2] = {k_out, v_out};
+  for (int i = 0; i < 2; ++i) {
+    if (!outs[i]) continue;
+    const uint4* base = (const uint4*)bufs[i] + sdvg::slot_offset(c, 0, slot) / 8;
+    if (c->head_dim == 128)
+      slot_read_kernel<128><<<blocks, kThreads, 0, (cudaStream_t)stream>>>(base, (uint4*)outs[i], c->block_tokens,
+                                                                          c->heads, stride);
+    else
+      slot_read_kernel<64><<<blocks, kThreads, 0, (cudaStream_t)stream>>>(base, (uint4*)outs[i], c->block_tokens,
+                                                                         c->heads, stride);
+    st = sdvg::cuda_status(cudaGetLastError());
+    if (st != SDVG_OK) return st;
+  }
+  return SDVG_OK;
+}
+
+}  // extern "C"

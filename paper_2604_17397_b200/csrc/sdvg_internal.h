@@ -1,0 +1,42 @@
+// Internal host-side declarations shared by the translation units of libsdvg.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "sdvg.h"
+
+struct sdvg_cache {
+  void* k_buf;
+  void* v_buf;
+  int slots, heads, block_tokens, head_dim;
+  int64_t next_block;
+  int64_t staged_block;                 // block whose provisional K/V sit in its slot, -1 if none
+  std::vector<int64_t> slot_block;      // slot -> committed block, -1 = empty
+};
+
+namespace sdvg {
+
+// Records a CUDA error for sdvg_last_cuda_error() and maps it to a status.
+int cuda_status(cudaError_t e);
+
+// SDVG_OK if the current device is compute capability 10.x (cached per device).
+int require_sm100();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline bool head_dim_ok(int d) { return d == 64 || d == 128; }
+
+// Element offset of (head, slot, token 0, dim 0) in a cache buffer laid out [heads][slots][tokens][dim].
+inline size_t slot_offset(const sdvg_cache* c, int head, int slot) {
+  return ((size_t)head * c->slots + slot) * (size_t)c->block_tokens * c->head_dim;
+}
+
+// Host-side ring bookkeeping shared by the commit entry points; returns a status and,
+// on success, the slot to write and (for SDVG_FINAL) the evicted block.
+int ring_begin_commit(sdvg_cache* c, int64_t block_index, int flags, int* slot);
+void ring_end_commit(sdvg_cache* c, int64_t block_index, int flags, int slot, int64_t* evicted);
+
+}  // namespace sdvg

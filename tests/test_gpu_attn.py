@@ -1,0 +1,164 @@
+"""GPU parity: sdvg_block_attn_fwd against the fp64 oracle on the same bits."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sdvg_oracle as O
+from paper_2604_17397_b200 import api, synth
+from gpu_utils import ATTN_MAX_ABS, ATTN_MEAN_ABS, ATTN_REL_RMS, attn_errors, to_bits, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def check(out_bits, ref, what=""):
+    mx, mean, rel = attn_errors(out_bits, ref)
+    assert mx <= ATTN_MAX_ABS and mean <= ATTN_MEAN_ABS, (what, mx, mean, rel)
+    assert rel <= ATTN_REL_RMS, (what, mx, mean, rel)
+    return mx, mean, rel
+
+
+def run_sequence(sh, nblocks, seed, staged, q_scale=1.0, with_lse=True, rows_per_head=None, full_heads=None):
+    """Generate nblocks blocks through a ring of sh.slots slots; compare every block's attention."""
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ws = api.attn_workspace()
+    rng = np.random.default_rng(seed)
+    for b in range(nblocks):
+        q = synth.block_tensor(sh, seed, b, 0, synth.Q, std=q_scale)
+        k = synth.block_tensor(sh, seed, b, 0, synth.K)
+        v = synth.block_tensor(sh, seed, b, 0, synth.V)
+        dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
+        out = torch.full_like(dq, float("nan"))
+        lse = torch.full((sh.heads, sh.block_tokens), float("nan"), device="cuda") if with_lse else None
+        if staged:
+            api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd(dq, None, None, cache, b, out, lse, sh.scale, ws)
+        else:
+            api.sdvg_block_attn_fwd(dq, dk, dv, cache, b, out, lse, sh.scale, ws)
+        assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+        got = to_bits(out)
+        if rows_per_head is None:
+            o_ref, lse_ref = O.block_attn_ref(q, k, v, ref, b, sh.scale)
+            check(got, o_ref, (sh.name, b, staged))
+            if with_lse:
+                assert np.allclose(lse.cpu().numpy(), lse_ref, rtol=0, atol=2e-3)
+        else:
+            for h in range(sh.heads):
+                rows = np.arange(sh.block_tokens) if (full_heads and h in full_heads) else \
+                    np.sort(rng.choice(sh.block_tokens, rows_per_head, replace=False))
+                o_ref, lse_ref = O.block_attn_ref(q, k, v, ref, b, sh.scale, heads=[h], rows=rows)
+                check(got[rows, h], o_ref[:, 0], (sh.name, b, h))
+                if with_lse:
+                    assert np.allclose(lse.cpu().numpy()[h, rows], lse_ref[0], rtol=0, atol=2e-3)
+        api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_FINAL)
+        ref.commit(b, k, v, O.FINAL)
+    cache.close()
+
+
+@pytest.mark.parametrize("staged", [False, True])
+def test_config1_tiny_every_fill_level(staged):
+    # 2 heads x d64, 64-token blocks, ring of 3: Lk = 64, 128, 192, then wrapped rings
+    run_sequence(synth.TINY, 5, 0, staged)
+
+
+@pytest.mark.parametrize("staged", [False, True])
+def test_d128_ragged_tiles_and_wraparound(staged):
+    # 2*5*23 = 230 tokens: two query tiles with a ragged tail, key segments with ragged ends
+    sh = synth.Shape("ragged128", heads=3, head_dim=128, frames=2, grid_h=5, grid_w=23, slots=3)
+    run_sequence(sh, 5, 41, staged)
+
+
+def test_d64_multi_tile():
+    sh = synth.Shape("ragged64", heads=2, head_dim=64, frames=3, grid_h=7, grid_w=19, slots=4)
+    run_sequence(sh, 6, 42, True)
+
+
+def test_peaky_logits_keep_the_absolute_tolerance():
+    # q scaled x4: softmax concentrates on few keys and outputs are O(1)
+    sh = synth.Shape("peaky", heads=2, head_dim=128, frames=1, grid_h=12, grid_w=25, slots=3)
+    run_sequence(sh, 4, 43, True, q_scale=4.0)
+
+
+def test_closed_forms_on_device():
+    sh = synth.Shape("cf", heads=2, head_dim=128, frames=1, grid_h=10, grid_w=20, slots=2)
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ws = api.attn_workspace()
+    k = synth.block_tensor(sh, 44, 0, 0, synth.K)
+    v = synth.block_tensor(sh, 44, 0, 0, synth.V)
+    q0 = np.zeros_like(k)
+    out = torch.empty_like(to_dev(k))
+    lse = torch.empty((sh.heads, sh.block_tokens), device="cuda")
+    api.sdvg_block_attn_fwd(to_dev(q0), to_dev(k), to_dev(v), cache, 0, out, lse, sh.scale, ws)
+    # q = 0: uniform weights, the output is the mean of V and lse = ln(Lk)
+    mean_v = O.bf16_to_f64(v).mean(axis=0)
+    got = O.bf16_to_f64(to_bits(out))
+    assert np.abs(got - mean_v[None]).max() <= 2e-3
+    assert np.allclose(lse.cpu().numpy(), np.log(sh.block_tokens), atol=1e-4)
+
+
+def test_config2_wan13b_shape_sampled_and_two_full_heads():
+    sh = synth.WAN_1_3B
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ws = api.attn_workspace()
+    for b in range(2):
+        k = synth.block_tensor(sh, 2, b, 0, synth.K)
+        v = synth.block_tensor(sh, 2, b, 0, synth.V)
+        api.sdvg_kv_commit(cache, to_dev(k), to_dev(v), b, api.SDVG_FINAL)
+        ref.commit(b, k, v, O.FINAL)
+    q, k, v = (synth.block_tensor(sh, 2, 2, 0, t) for t in (synth.Q, synth.K, synth.V))
+    out = torch.empty_like(to_dev(q))
+    api.sdvg_kv_commit(cache, to_dev(k), to_dev(v), 2, api.SDVG_STAGE)
+    api.sdvg_block_attn_fwd(to_dev(q), None, None, cache, 2, out, None, sh.scale, ws)
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    got = to_bits(out)
+    rng = np.random.default_rng(2)
+    for h in range(sh.heads):
+        rows = np.arange(sh.block_tokens) if h in (0, 11) else np.sort(rng.choice(sh.block_tokens, 96, replace=False))
+        o_ref, _ = O.block_attn_ref(q, k, v, ref, 2, sh.scale, heads=[h], rows=rows)
+        check(got[rows, h], o_ref[:, 0], ("wan1.3b", h))
+
+
+def test_config3_wan14b_shape_fused_prologue_cache_bits_and_sampled_attention():
+    sh = synth.WAN_14B
+    grid = (sh.frames, sh.grid_h, sh.grid_w)
+    tabf = 7 * sh.frames
+    ref_tab = O.rope_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w)
+    dev_tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ws = api.attn_workspace()
+    pool = synth.TensorPool(sh, 3)
+    for b in range(6):
+        k, v = pool.get(b, 0, synth.K), pool.get(b, 0, synth.V)
+        ev = api.sdvg_rope3d_qk_commit(cache, None, to_dev(k), to_dev(v), None, None, grid, b * sh.frames, dev_tab,
+                                       tabf, b, api.SDVG_FINAL)
+        assert ev == -1
+        ref.commit(b, O.rope_bitspec(k, grid, b * sh.frames, ref_tab, tabf), v, O.FINAL)
+    b = 6
+    q, k, v = (synth.block_tensor(sh, 3, b, 0, t) for t in (synth.Q, synth.K, synth.V))
+    dq = to_dev(q)
+    q_r = torch.empty_like(dq)
+    api.sdvg_rope3d_qk_commit(cache, dq, to_dev(k), to_dev(v), q_r, None, grid, b * sh.frames, dev_tab, tabf, b,
+                              api.SDVG_STAGE)
+    out = torch.empty_like(dq)
+    lse = torch.empty((sh.heads, sh.block_tokens), device="cuda")
+    api.sdvg_block_attn_fwd(q_r, None, None, cache, b, out, lse, sh.scale, ws)
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    qr_ref = O.rope_bitspec(q, grid, b * sh.frames, ref_tab, tabf)
+    kr_ref = O.rope_bitspec(k, grid, b * sh.frames, ref_tab, tabf)
+    assert np.array_equal(to_bits(q_r), qr_ref)
+    # cache contents, bit for bit, all 7 slots (slot 6 holds the staged block)
+    for s in range(6):
+        gk, gv = cache.read_block(s)
+        assert np.array_equal(to_bits(gk), ref.k[s]) and np.array_equal(to_bits(gv), ref.v[s])
+    gk, gv = cache.read_block(6)
+    assert np.array_equal(to_bits(gk), kr_ref) and np.array_equal(to_bits(gv), v)
+    got = to_bits(out)
+    rng = np.random.default_rng(3)
+    lse_h = lse.cpu().numpy()
+    for h in range(sh.heads):
+        rows = np.arange(sh.block_tokens) if h in (0, 39) else np.sort(rng.choice(sh.block_tokens, 64, replace=False))
+        o_ref, lse_ref = O.block_attn_ref(qr_ref, kr_ref, v, ref, b, sh.scale, heads=[h], rows=rows)
+        check(got[rows, h], o_ref[:, 0], ("wan14b", h))
+        assert np.allclose(lse_h[h, rows], lse_ref[0], rtol=0, atol=2e-3)
