@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the SDVG hot path on B200: one denoise step at the Wan-14B target shape.
+
+A step is one pass of the whole path over one block: fused 3D-RoPE + stage of K/V into the
+ring -> block attention of 4680 queries against the full 7-slot ring (32760 keys) -> final
+commit of the block -> routing of a batch of per-frame scores.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 14b|1.3b]
+
+--impl reference times the CPU oracle (the only other place the oracle runs) on a bounded
+sample of the same workload and prints the same line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "block-attn TFLOP/s per denoise step @14B shape (% bf16 peak); KV-commit GB/s"
+ROUTE_BLOCKS = 1003 * 9          # the paper's evaluation volume: 1003 videos x 9 blocks (Sec. 4.1)
+ROUTE_FRAMES = 12
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def workload_shape(name: str):
+    from paper_2604_17397_b200 import synth
+    return {"14b": synth.WAN_14B, "1.3b": synth.WAN_1_3B, "tiny": synth.TINY}[name]
+
+
+def attn_flops(sh, lk: int) -> float:
+    """Algorithmic FLOPs of one attention call: QK^T and PV, 2 flops per multiply-add, no padding."""
+    return 4.0 * sh.block_tokens * lk * sh.head_dim * sh.heads
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 100 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str | None):
+        self.uuid, self.proc, self.path = uuid, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.uuid:
+                cmd.insert(1, f"--id={self.uuid}")
+            self.proc = subprocess.Popen(cmd, stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        with open(self.path) as f:
+            for line in f:
+                c = [x.strip() for x in line.split(",")]
+                if len(c) >= 7:
+                    rows.append(c)
+        os.unlink(self.path)
+        if not rows:
+            return out
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+        out.update(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=float(rows[0][1]), reasons=reasons,
+                   samples=len(rows), power_w_max=max(float(r[2]) for r in rows))
+        return out
+
+
+# --------------------------------------------------------------------------- reference arm / cpu baseline
+
+def oracle_sample(sh, heads_sampled: int, lk_blocks: int, seed: int = 3):
+    """Inputs of the oracle's bounded sample: `heads_sampled` heads of one full-window step."""
+    from paper_2604_17397_b200 import synth
+    sub = synth.Shape(sh.name + "-sample", heads_sampled, sh.head_dim, sh.frames, sh.grid_h, sh.grid_w, sh.slots)
+    q = synth.block_tensor(sub, seed, lk_blocks - 1, 0, synth.Q)
+    ks = [synth.block_tensor(sub, seed, b, 0, synth.K) for b in range(lk_blocks)]
+    vs = [synth.block_tensor(sub, seed, b, 0, synth.V) for b in range(lk_blocks)]
+    scores = synth.normal_scores(ROUTE_BLOCKS, ROUTE_FRAMES, -0.5, 0.6, seed)
+    return sub, q, ks, vs, scores
+
+
+def oracle_step(sub, q, ks, vs, scores, tab, tabf):
+    """One pass of the path through the oracle on the sample (rope -> stage -> attention -> commit -> route)."""
+    from oracle import sdvg_oracle as O
+    grid = (sub.frames, sub.grid_h, sub.grid_w)
+    n = len(ks)
+    cache = O.RingCacheRef(sub.slots, sub.heads, sub.block_tokens, sub.head_dim)
+    for b in range(n - 1):
+        cache.commit(b, ks[b], vs[b], O.FINAL)           # window prepared outside the timed part
+    t0 = time.perf_counter()
+    fo = (n - 1) * sub.frames
+    qr = O.rope_bitspec(q, grid, fo, tab, tabf)
+    kr = O.rope_bitspec(ks[-1], grid, fo, tab, tabf)
+    cache.commit(n - 1, kr, vs[-1], O.STAGE)
+    O.block_attn_ref(qr, kr, vs[-1], cache, n - 1, sub.scale)
+    cache.commit(n - 1, kr, vs[-1], O.FINAL)
+    O.route_ref(scores.reshape(-1)[: 2000 * ROUTE_FRAMES], None, 2000, ROUTE_FRAMES, 0, -0.7)
+    return time.perf_counter() - t0
+
+
+def run_oracle(sh, steps: int, warmup: int, heads_sampled: int):
+    from oracle import sdvg_oracle as O
+    lk_blocks = sh.slots
+    sub, q, ks, vs, scores = oracle_sample(sh, heads_sampled, lk_blocks)
+    tabf = lk_blocks * sh.frames
+    tab = O.rope_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w)
+    for _ in range(warmup):
+        oracle_step(sub, q, ks, vs, scores, tab, tabf)
+    times = [oracle_step(sub, q, ks, vs, scores, tab, tabf) for _ in range(steps)]
+    sec = float(np.mean(times))
+    flops = attn_flops(sub, lk_blocks * sh.block_tokens)
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        pass
+    sample = (f"{heads_sampled} of {sh.heads} heads of one full-window step ({sh.block_tokens} queries x "
+              f"{lk_blocks * sh.block_tokens} keys, d{sh.head_dim}), rope + stage + attention + commit on those "
+              f"heads, route on 2000 of {ROUTE_BLOCKS} blocks")
+    return {"value": flops / sec / 1e12, "unit": "TFLOP/s", "cores": int(cores), "kind": "oracle",
+            "sample": sample, "sec_per_sample_step": sec}
+
+
+# --------------------------------------------------------------------------- our arm
+
+class Step:
+    """Device-resident state of the benchmarked step and the calls that make one step."""
+
+    def __init__(self, sh, device, max_steps: int, seed: int = 3):
+        import torch
+        from paper_2604_17397_b200 import api, synth
+        self.torch, self.api, self.sh = torch, api, sh
+        self.grid = (sh.frames, sh.grid_h, sh.grid_w)
+        self.tabf = (sh.slots + max_steps + 2) * sh.frames
+        self.tab = api.sdvg_rope3d_table(sh.head_dim, self.tabf, sh.grid_h, sh.grid_w).to(device)
+        self.cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device)
+        self.ws = api.attn_workspace(device=device)
+        pool = synth.TensorPool(sh, seed, n=3)
+
+        def dev(bits):
+            return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+
+        self.host = [torch.from_numpy(pool.get(0, 0, t).view(np.int16)).view(torch.bfloat16).pin_memory()
+                     for t in (synth.Q, synth.K, synth.V)]
+        self.q, self.k, self.v = (h.to(device) for h in self.host)
+        self.q_r = torch.empty_like(self.q)
+        self.k_r = torch.empty_like(self.k)
+        self.out = torch.empty_like(self.q)
+        self.out_host = torch.empty_like(self.q, device="cpu").pin_memory()
+        scores = synth.normal_scores(ROUTE_BLOCKS, ROUTE_FRAMES, -0.5, 0.6, seed)
+        self.scores_host = torch.from_numpy(scores.reshape(-1)).pin_memory()
+        self.scores = self.scores_host.to(device)
+        self.accept = torch.empty(ROUTE_BLOCKS, dtype=torch.uint8, device=device)
+        self.qmin = torch.empty(ROUTE_BLOCKS, dtype=torch.float32, device=device)
+        self.accept_host = torch.empty(ROUTE_BLOCKS, dtype=torch.uint8).pin_memory()
+        self.block = 0
+        for _ in range(sh.slots - 1):                      # fill the window: slots-1 committed blocks
+            api.sdvg_rope3d_qk_commit(self.cache, None, self.k, self.v, None, None, self.grid,
+                                      self.block * sh.frames, self.tab, self.tabf, self.block, api.SDVG_FINAL)
+            self.block += 1
+        self.attn_events = []
+        self.lk = sh.slots * sh.block_tokens
+
+    def step(self, time_attention: bool = False):
+        api, sh, b = self.api, self.sh, self.block
+        api.sdvg_rope3d_qk_commit(self.cache, self.q, self.k, self.v, self.q_r, self.k_r, self.grid, b * sh.frames,
+                                  self.tab, self.tabf, b, api.SDVG_STAGE)
+        if time_attention:
+            e0, e1 = self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+            e0.record()
+        api.sdvg_block_attn_fwd(self.q_r, None, None, self.cache, b, self.out, None, sh.scale, self.ws)
+        if time_attention:
+            e1.record()
+            self.attn_events.append((e0, e1))
+        api.sdvg_kv_commit(self.cache, self.k_r, self.v, b, api.SDVG_FINAL)
+        api.sdvg_route(self.scores, None, ROUTE_BLOCKS, ROUTE_FRAMES, 0, -0.7, self.accept, self.qmin, None)
+        self.block += 1
+    LAUNCHES_PER_STEP = 4          # rope+stage, attention, commit, route
+
+    def step_e2e(self):
+        for d, h in zip((self.q, self.k, self.v), self.host):
+            d.copy_(h, non_blocking=True)
+        self.scores.copy_(self.scores_host, non_blocking=True)
+        self.step()
+        self.out_host.copy_(self.out, non_blocking=True)
+        self.accept_host.copy_(self.accept, non_blocking=True)
+
+    def e2e_bytes(self):
+        h2d = sum(h.numel() * h.element_size() for h in self.host) + self.scores_host.numel() * 4
+        d2h = self.out_host.numel() * 2 + self.accept_host.numel()
+        return h2d, d2h
+
+    def hbm_bytes(self):
+        """Algorithmic HBM bytes of the three streaming kernels of one step."""
+        t = self.sh.block_tokens * self.sh.heads * self.sh.head_dim * 2
+        return {"rope_stage": 7 * t,      # read q,k,v; write q', k' (logical), k' and v (ring)
+                "commit": 4 * t,          # read k', v; write both into the ring
+                "route": ROUTE_BLOCKS * (ROUTE_FRAMES * 4 + 5)}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_17397_b200 import api, dist_util
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    api.lib()
+    sh = workload_shape(args.workload)
+    st = Step(sh, device, max_steps=2 * (args.steps + args.warmup) + 8)
+    pk = peaks()
+
+    for _ in range(args.warmup):
+        st.step()
+    torch.cuda.synchronize()
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid if rank == 0 else None)
+    if rank == 0:
+        sampler.start()
+    dist_util.barrier(world)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        st.step(time_attention=True)
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier(world)
+    ms_total = dist_util.max_over_ranks(e0.elapsed_time(e1), world, device)
+    clocks = sampler.stop() if rank == 0 else None
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in st.attn_events]))
+    assert api.sdvg_block_attn_status(st.ws) == api.SDVG_OK, "attention kernel reported a timeout"
+
+    # the streaming kernels, each timed alone (their inputs and outputs exceed L2 at this shape)
+    def time_call(fn, n=10):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    hb = st.hbm_bytes()
+    blk = st.block
+    t_rope = time_call(lambda: api.sdvg_rope3d_qk_commit(st.cache, st.q, st.k, st.v, st.q_r, st.k_r, st.grid,
+                                                         blk * sh.frames, st.tab, st.tabf, blk, api.SDVG_STAGE))
+    t_commit = time_call(lambda: api.sdvg_kv_commit(st.cache, st.k_r, st.v, blk, api.SDVG_STAGE))
+    t_route = time_call(lambda: api.sdvg_route(st.scores, None, ROUTE_BLOCKS, ROUTE_FRAMES, 0, -0.7, st.accept,
+                                               st.qmin, None))
+
+    # end to end through the same calls with host buffers: H2D of q,k,v,scores and D2H of out, accept per step
+    for _ in range(2):
+        st.step_e2e()
+    torch.cuda.synchronize()
+    dist_util.barrier(world)
+    n_e2e = max(3, args.steps // 2)
+    e0.record()
+    for _ in range(n_e2e):
+        st.step_e2e()
+    e1.record()
+    torch.cuda.synchronize()
+    ms_e2e = dist_util.max_over_ranks(e0.elapsed_time(e1), world, device) / n_e2e
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    flops = attn_flops(sh, st.lk)
+    ms_step = ms_total / args.steps
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    attn_tflops = flops / (attn_ms * 1e-3) / 1e12
+    h2d, d2h = st.e2e_bytes()
+    cpu = run_oracle(sh, steps=1, warmup=0, heads_sampled=2) if world == 1 and not args.no_cpu_baseline else None
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{sh.name}: {sh.heads} heads x d{sh.head_dim}, {sh.block_tokens}-token block vs "
+                               f"{sh.slots}-slot ring ({st.lk} keys), fused rope+stage, attention, final commit, "
+                               f"route of {ROUTE_BLOCKS}x{ROUTE_FRAMES} scores",
+                   "cache": "inputs larger than L2 (ring 2 x %.0f MB, q/k/v 3 x %.0f MB per step); no flush"
+                            % (st.cache.slots * sh.block_tokens * sh.heads * sh.head_dim * 2 / 1e6,
+                               sh.block_tokens * sh.heads * sh.head_dim * 2 / 1e6),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks,
+        "e2e": {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": Step.LAUNCHES_PER_STEP * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "sdvg_block_attn_fwd", "achieved": attn_tflops,
+                     "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": attn_tflops / pk["bf16_tflops"],
+                     "frac_of_sustained_peak": attn_tflops / pk["bf16_tflops_sustained"],
+                     "frac_of_nominal_2250": attn_tflops / 2250.0, "peak_source": pk["source"],
+                     "ms_per_launch": attn_ms, "traffic": None},
+        "hbm_kernels": {
+            "peak_gbs": pk["hbm_gbs"],
+            "rope_stage": {"ms": t_rope, "gbs": hb["rope_stage"] / t_rope / 1e6,
+                           "frac": hb["rope_stage"] / t_rope / 1e6 / pk["hbm_gbs"]},
+            "kv_commit": {"ms": t_commit, "gbs": hb["commit"] / t_commit / 1e6,
+                          "frac": hb["commit"] / t_commit / 1e6 / pk["hbm_gbs"]},
+            "route": {"us": t_route * 1e3, "gbs": hb["route"] / t_route / 1e6}},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sh = workload_shape(args.workload)
+    steps = max(1, min(args.steps, 3))
+    cpu = run_oracle(sh, steps=steps, warmup=min(args.warmup, 1), heads_sampled=2)
+    lk = sh.slots * sh.block_tokens
+    line = {"impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": "TFLOP/s",
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": min(args.warmup, 1),
+            "ms_per_step": cpu["sec_per_sample_step"] * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{sh.name}: bounded sample of the {sh.block_tokens}-query x {lk}-key step "
+                                   f"({cpu['sample']})"},
+            "cpu_baseline": cpu,
+            "e2e": {"value": cpu["value"], "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="14b", choices=["14b", "1.3b", "tiny"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
