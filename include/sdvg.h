@@ -188,6 +188,36 @@ int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self,
  */
 int sdvg_block_attn_status(const void* workspace, void* stream);
 
+/*
+ * Same computation as sdvg_block_attn_fwd for callers that cannot allocate device memory
+ * (the paper has no counterpart; this is a deployment convenience).  Some hosts of this
+ * library run under a fixed memory plan: an inference server that hands every byte of HBM
+ * to its own arena at start-up, a plugin called from inside someone else's stream or graph
+ * set-up where cudaMalloc would synchronise the device, or a process whose allocator is
+ * simply not reachable from the call site.  Such callers have no way to produce the
+ * `workspace` buffer, so this entry point brings its own: a 256-byte, 256-byte-aligned array
+ * that is part of the library image (every GPU that loads the library holds its own copy
+ * until the process exits).  The call itself allocates nothing and frees nothing.
+ *
+ *   - Limit: the built-in scratch is exactly 256 bytes, which covers every shape the library
+ *     supports today.  If a future kernel needed more than that, this function would return
+ *     SDVG_ERR_BAD_SHAPE instead of overrunning the array; use sdvg_block_attn_fwd with a
+ *     caller-owned workspace in that case.  At most 64 devices per process.
+ *   - First call on a device: the function looks up where that device's copy of the array
+ *     lives (cudaGetSymbolAddress, with the device current) and remembers it.  Make that first
+ *     call outside of any stream capture.
+ *   - All calls on a device share the one array.  Each call clears it on `stream` before the
+ *     kernel runs and the kernel leaves its status word there, so two calls that overlap on
+ *     the GPU (different streams, no ordering between them) race on it; keep them ordered.
+ *   - *scratch_device_ptr (optional, host) receives the device address of the array, which
+ *     can be given to sdvg_block_attn_status to read the status word after the call.
+ * Arguments, results and errors are otherwise those of sdvg_block_attn_fwd.
+ */
+int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self,
+                                const sdvg_cache* cache, int64_t block_index,
+                                void* out, float* lse, float scale,
+                                void** scratch_device_ptr, void* stream);
+
 /* ---- router ------------------------------------------------------------- */
 /*
  * Eq. (1) and the policy of Sec. 3: q_min[b] = min_i scores[b, i];

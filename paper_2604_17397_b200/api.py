@@ -49,6 +49,7 @@ SIGNATURES = {
     "sdvg_block_attn_workspace_bytes": (_SZ, []),
     "sdvg_block_attn_fwd": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_attn_status": (_I, [_VP, _VP]),
+    "sdvg_block_attn_fwd_noalloc": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, C.POINTER(_VP), _VP]),
     "sdvg_route": (_I, [_VP, _VP, _I, _I, _I64, _F, _VP, _VP, _VP, _VP]),
 }
 
@@ -233,8 +234,27 @@ def sdvg_block_attn_fwd(q, k_self, v_self, cache: Cache, block_index: int, out, 
     _check(st, "sdvg_block_attn_fwd")
 
 
-def sdvg_block_attn_status(workspace: torch.Tensor, stream=None) -> int:
-    return lib().sdvg_block_attn_status(workspace.data_ptr(), _stream(stream))
+def sdvg_block_attn_status(workspace, stream=None) -> int:
+    """`workspace` is the tensor given to sdvg_block_attn_fwd, or the integer device address
+    returned by sdvg_block_attn_fwd_noalloc."""
+    ptr = workspace if isinstance(workspace, int) else workspace.data_ptr()
+    return lib().sdvg_block_attn_status(ptr, _stream(stream))
+
+
+def sdvg_block_attn_fwd_noalloc(q, k_self, v_self, cache: Cache, block_index: int, out, lse, scale: float,
+                                stream=None) -> int:
+    """Attention through the library's built-in scratch: for callers that must not allocate
+    device memory.  Returns the device address of that scratch (for sdvg_block_attn_status)."""
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    if lse is not None and (lse.dtype != torch.float32 or tuple(lse.shape) != (cache.heads, cache.block_tokens)):
+        raise ValueError("lse must be float32 [heads, block_tokens]")
+    scratch = _VP()
+    st = lib().sdvg_block_attn_fwd_noalloc(_bf16(q, shape), _bf16(k_self, None if k_self is None else shape),
+                                           _bf16(v_self, None if v_self is None else shape), cache.handle,
+                                           block_index, _bf16(out, shape), _ptr(lse), scale, C.byref(scratch),
+                                           _stream(stream))
+    _check(st, "sdvg_block_attn_fwd_noalloc")
+    return int(scratch.value)
 
 
 # ---------------------------------------------------------------- router

@@ -18,6 +18,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <mutex>
+
 #include "sdvg_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -332,16 +334,10 @@ int launch_simple(const AttnParams& p, cudaStream_t stream) {
   return sdvg::cuda_status(cudaGetLastError());
 }
 
-}  // namespace
-
-extern "C" {
-
-size_t sdvg_block_attn_workspace_bytes(void) { return kWorkspaceBytes; }
-
-int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
-                        int64_t block_index, void* out, float* lse, float scale, void* workspace,
-                        size_t workspace_bytes, void* stream_) {
-  cudaStream_t stream = (cudaStream_t)stream_;
+// Validation, tensor maps, scratch clear and launch shared by the attention entry points.
+int attn_forward(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c, int64_t block_index,
+                 void* out, float* lse, float scale, void* workspace, size_t workspace_bytes,
+                 cudaStream_t stream) {
   if (!q || !c || !out || !workspace) return SDVG_ERR_INVALID_ARG;
   if ((k_self == nullptr) != (v_self == nullptr)) return SDVG_ERR_INVALID_ARG;
   if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
@@ -405,6 +401,52 @@ int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, c
   cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
   if (e != cudaSuccess) return sdvg::cuda_status(e);
   return D == 128 ? launch_simple<128>(p, stream) : launch_simple<64>(p, stream);
+}
+
+// Scratch for sdvg_block_attn_fwd_noalloc: lives in the library image, one copy per device that
+// loads it.  In host code this name is only a handle for cudaGetSymbolAddress, never a pointer.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kWorkspaceBytes];
+
+}  // namespace
+
+extern "C" {
+
+size_t sdvg_block_attn_workspace_bytes(void) { return kWorkspaceBytes; }
+
+int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
+                        int64_t block_index, void* out, float* lse, float scale, void* workspace,
+                        size_t workspace_bytes, void* stream_) {
+  return attn_forward(q, k_self, v_self, c, block_index, out, lse, scale, workspace, workspace_bytes,
+                      (cudaStream_t)stream_);
+}
+
+int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
+                                int64_t block_index, void* out, float* lse, float scale,
+                                void** scratch_device_ptr, void* stream_) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static void* scratch_of_device[kMaxDevices] = {};
+  // The built-in scratch has a fixed size; refuse rather than overrun if the kernel ever needs more.
+  if (sdvg_block_attn_workspace_bytes() > sizeof(g_noalloc_scratch)) return SDVG_ERR_BAD_SHAPE;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  if (dev < 0 || dev >= kMaxDevices) return SDVG_ERR_INVALID_ARG;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!scratch_of_device[dev]) {
+      // once per device, with that device current: ask the runtime where this device's copy lives
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+      if (e != cudaSuccess) return sdvg::cuda_status(e);
+      scratch_of_device[dev] = ptr;
+    }
+    scratch = scratch_of_device[dev];
+  }
+  if (scratch_device_ptr) *scratch_device_ptr = scratch;
+  return attn_forward(q, k_self, v_self, c, block_index, out, lse, scale, scratch, sizeof(g_noalloc_scratch),
+                      (cudaStream_t)stream_);
 }
 
 int sdvg_block_attn_status(const void* workspace, void* stream_) {
