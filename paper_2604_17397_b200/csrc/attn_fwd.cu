@@ -17,6 +17,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include <mutex>
 
@@ -55,19 +56,29 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+
 struct WaitCtx {
   volatile int* abort_flag;            // shared
   unsigned int* status;                // global
-  uint64_t t0;
+  uint64_t t0;                         // unused by the wait itself; kept for diagnostics
 };
 
-// Bounded mbarrier wait.  Returns false once the CTA is aborting.
+// Bounded mbarrier wait: gives up kWaitLimitNs after its own first slow poll.  Returns false once
+// the CTA is aborting.
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, const WaitCtx& c) {
+  uint64_t start = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0xff) == 0xff) {
       if (*c.abort_flag) return false;
-      if (globaltimer_ns() - c.t0 > kWaitLimitNs) {
+      const uint64_t now = globaltimer_ns();
+      if (start == 0) start = now;
+      if (now - start > kWaitLimitNs) {
         *c.abort_flag = 1;
         atomicExch(c.status, (unsigned)SDVG_ERR_TIMEOUT);
         return false;
@@ -286,6 +297,8 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+#include "attn_fwd_ws.cuh"
+
 // ---- host side -------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -332,6 +345,34 @@ int launch_simple(const AttnParams& p, cudaStream_t stream) {
   dim3 grid((p.tokens + kTileM - 1) / kTileM, p.heads);
   attn_fwd_simple_kernel<D><<<grid, 128, SimpleSmem<D>::kDynamic, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
+}
+
+template <int D>
+int launch_ws(const AttnParams& p, cudaStream_t stream) {
+  static bool configured = false;
+  static int sms = 0;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         WsCfg<D>::kDynamic);
+    if (e != cudaSuccess) return sdvg::cuda_status(e);
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    configured = true;
+  }
+  const WsSchedule sched(p.tokens, p.heads);
+  const int grid = sched.num_virtual < sms ? sched.num_virtual : sms;
+  attn_fwd_ws_kernel<D><<<grid, WsCfg<D>::kThreads, WsCfg<D>::kDynamic, stream>>>(p);
+  return sdvg::cuda_status(cudaGetLastError());
+}
+
+bool use_simple_kernel() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SDVG_ATTN_KERNEL");
+    v = (e && e[0] == 's') ? 1 : 0;
+  }
+  return v == 1;
 }
 
 // Validation, tensor maps, scratch clear and launch shared by the attention entry points.
@@ -400,7 +441,8 @@ int attn_forward(const void* q, const void* k_self, const void* v_self, const sd
 #endif
   cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
   if (e != cudaSuccess) return sdvg::cuda_status(e);
-  return D == 128 ? launch_simple<128>(p, stream) : launch_simple<64>(p, stream);
+  if (use_simple_kernel()) return D == 128 ? launch_simple<128>(p, stream) : launch_simple<64>(p, stream);
+  return D == 128 ? launch_ws<128>(p, stream) : launch_ws<64>(p, stream);
 }
 
 // Scratch for sdvg_block_attn_fwd_noalloc: lives in the library image, one copy per device that
