@@ -29,6 +29,7 @@ if ROOT not in sys.path:
 METRIC = "block-attn TFLOP/s per denoise step @14B shape (% bf16 peak); KV-commit GB/s"
 ROUTE_BLOCKS = 1003 * 9          # the paper's evaluation volume: 1003 videos x 9 blocks (Sec. 4.1)
 ROUTE_FRAMES = 12
+CPU_SAMPLE_HEADS = 12           # heads of one step the CPU oracle is timed on (about 10-20 s of host work)
 
 
 def peaks():
@@ -52,7 +53,7 @@ def attn_flops(sh, lk: int) -> float:
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 100 ms while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons sampled every 20 ms while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -64,7 +65,7 @@ class ClockSampler:
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
-            cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+            cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"]
             if self.uuid:
                 cmd.insert(1, f"--id={self.uuid}")
             self.proc = subprocess.Popen(cmd, stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
@@ -316,7 +317,7 @@ def run_ours(args):
     value = world * flops / (ms_step * 1e-3) / 1e12
     attn_tflops = flops / (attn_ms * 1e-3) / 1e12
     h2d, d2h = st.e2e_bytes()
-    cpu = run_oracle(sh, steps=1, warmup=0, heads_sampled=2) if world == 1 and not args.no_cpu_baseline else None
+    cpu = run_oracle(sh, steps=1, warmup=0, heads_sampled=CPU_SAMPLE_HEADS) if world == 1 and not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -357,7 +358,7 @@ def run_reference(args):
         return
     sh = workload_shape(args.workload)
     steps = max(1, min(args.steps, 3))
-    cpu = run_oracle(sh, steps=steps, warmup=min(args.warmup, 1), heads_sampled=2)
+    cpu = run_oracle(sh, steps=steps, warmup=min(args.warmup, 1), heads_sampled=min(CPU_SAMPLE_HEADS, sh.heads))
     lk = sh.slots * sh.block_tokens
     line = {"impl": "reference", "metric": METRIC, "value": cpu["value"], "unit": "TFLOP/s",
             "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": min(args.warmup, 1),
@@ -373,7 +374,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="14b", choices=["14b", "1.3b", "tiny"])

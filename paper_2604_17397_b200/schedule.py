@@ -1,0 +1,126 @@
+"""Per-block speculative schedule (Sec. 3 "Inference flow", Fig. 2) on the device.
+
+Host glue only: it strings the library's entry points together in the order the
+paper gives and takes the accept/reject branch on the host.  For every block b
+
+  1. the drafter takes ``steps`` denoise steps; each step is one fused
+     rope + stage call and one attention call against the drafter ring K^D;
+  2. the drafter's final K/V of the block are committed to K^D unconditionally
+     (the drafter always conditions on its own earlier outputs);
+  3. the router scores the block (worst frame against tau, global block 0 is
+     always rejected);
+  4. accepted: the target-shaped K/V of the draft block are committed to the
+     target ring K^T.  Rejected: the target takes ``steps`` steps of its own
+     against K^T and commits the K/V of the regenerated block.
+
+K^D and K^T are independent rings with their own shapes and window sizes.
+The tensors of every call come from a ``provider`` callback, so the same
+function drives synthetic traces and a real model.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Callable, Optional
+
+import numpy as np
+import torch
+
+from . import api
+
+
+@dataclass
+class ModelState:
+    """Everything one model (drafter or target) needs for its steps."""
+    cache: api.Cache
+    grid: tuple                    # (latent frames per block, grid rows, grid columns)
+    table: torch.Tensor            # device (cos, sin) table built for tab_frames frame positions
+    tab_frames: int
+    scale: float
+    workspace: torch.Tensor = None
+
+    def __post_init__(self):
+        if self.workspace is None:
+            self.workspace = api.attn_workspace(device=self.table.device)
+        shape = (self.cache.block_tokens, self.cache.heads, self.cache.head_dim)
+        dev = self.table.device
+        self.q_roped = torch.empty(shape, dtype=torch.bfloat16, device=dev)
+        self.k_roped = torch.empty(shape, dtype=torch.bfloat16, device=dev)
+        self.out = torch.empty(shape, dtype=torch.bfloat16, device=dev)
+
+    @property
+    def frames(self) -> int:
+        return self.grid[0]
+
+
+@dataclass
+class TraceResult:
+    accept: np.ndarray
+    q_min: np.ndarray
+    drafter_evicted: list = field(default_factory=list)
+    target_evicted: list = field(default_factory=list)
+    drafter_attn_calls: int = 0
+    target_attn_calls: int = 0
+    target_source: list = field(default_factory=list)     # per block: "accepted" or "regenerated"
+
+
+def _denoise(model: str, m: ModelState, block: int, steps: int, provider, on_attention) -> int:
+    for s in range(steps):
+        q, k, v = provider(model, block, "step", s)
+        api.sdvg_rope3d_qk_commit(m.cache, q, k, v, m.q_roped, None, m.grid, block * m.frames, m.table,
+                                  m.tab_frames, block, api.SDVG_STAGE)
+        api.sdvg_block_attn_fwd(m.q_roped, None, None, m.cache, block, m.out, None, m.scale, m.workspace)
+        if on_attention is not None:
+            on_attention(model, block, s, m.q_roped, m.out)
+    return steps
+
+
+def _commit_clean(m: ModelState, block: int, k, v) -> int:
+    """Rope the block's final K and write it with V into the ring (SDVG_FINAL)."""
+    return api.sdvg_rope3d_qk_commit(m.cache, None, k, v, None, None, m.grid, block * m.frames, m.table,
+                                     m.tab_frames, block, api.SDVG_FINAL)
+
+
+def run_schedule(num_blocks: int, steps: int, scores: torch.Tensor, tau: float,
+                 drafter: ModelState, target: ModelState,
+                 provider: Callable, first_block_index: int = 0,
+                 on_attention: Optional[Callable] = None) -> TraceResult:
+    """Generate ``num_blocks`` blocks with the drafter/router/target flow.
+
+    scores    device fp32 [num_blocks, frames]: the per-frame reward of every draft block
+              (in a real system they appear one block at a time; routing here is also
+              done one block at a time, with the block's global index)
+    provider  ``provider(model, block, kind, step)`` -> (q, k, v) device bf16 tensors of the
+              model's shape; kind is "step" (one denoise step), "clean" (the model's final
+              K/V, q is None) or "accepted" (target-shaped K/V of an accepted draft block)
+    on_attention  optional ``f(model, block, step, q_roped, out)`` called after each
+              attention launch (the tensors are reused by the next step)
+    The accept decision is read back to the host once per block, which is the only
+    synchronisation point of the flow.
+    """
+    if scores.dtype != torch.float32 or scores.dim() != 2 or scores.shape[0] != num_blocks:
+        raise ValueError("scores must be float32 [num_blocks, frames]")
+    frames = scores.shape[1]
+    dev = scores.device
+    accept_d = torch.zeros(num_blocks, dtype=torch.uint8, device=dev)
+    qmin_d = torch.zeros(num_blocks, dtype=torch.float32, device=dev)
+    res = TraceResult(accept=np.zeros(num_blocks, dtype=np.uint8), q_min=np.zeros(num_blocks, dtype=np.float32))
+    flat = scores.reshape(-1)
+    for i in range(num_blocks):
+        b = first_block_index + i
+        res.drafter_attn_calls += _denoise("drafter", drafter, b, steps, provider, on_attention)
+        _, k, v = provider("drafter", b, "clean", 0)
+        res.drafter_evicted.append(_commit_clean(drafter, b, k, v))
+        api.sdvg_route(flat[i * frames:(i + 1) * frames], None, 1, frames, b, tau, accept_d[i:i + 1],
+                       qmin_d[i:i + 1], None)
+        accepted = bool(accept_d[i].item())
+        if accepted:
+            _, k, v = provider("target", b, "accepted", 0)
+            res.target_source.append("accepted")
+        else:
+            res.target_attn_calls += _denoise("target", target, b, steps, provider, on_attention)
+            _, k, v = provider("target", b, "clean", 0)
+            res.target_source.append("regenerated")
+        res.target_evicted.append(_commit_clean(target, b, k, v))
+    res.accept = accept_d.cpu().numpy()
+    res.q_min = qmin_d.cpu().numpy()
+    return res

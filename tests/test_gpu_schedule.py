@@ -1,0 +1,202 @@
+"""GPU parity of the whole per-block flow at the full model shapes.
+
+Config 4: the 14B target generates 9 blocks (7 fill the ring, 2 more evict), 4 denoise steps
+each; attention is checked on sampled rows at every fill level and step, the written ring slot
+bit for bit after every commit.
+Config 5: the drafter/router/target schedule over 16 blocks at the 1.3B and 14B shapes; accept
+vectors, q_min bits, eviction logs, slot maps and the final contents of both rings must equal the
+oracle's exactly, attention is checked on sampled rows at sampled points of the trace.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sdvg_oracle as O
+from paper_2604_17397_b200 import api, schedule, synth
+from gpu_utils import ATTN_MAX_ABS, ATTN_MEAN_ABS, ATTN_REL_RMS, attn_errors, to_bits, to_dev
+
+pytestmark = pytest.mark.gpu
+
+STEPS = 4                      # denoise steps per block (Sec. 4.1 "Models")
+
+
+class Provider:
+    """(model, block, kind, step) -> bf16 bits of (q, k, v), the same for the oracle and the GPU."""
+
+    SRC = {("drafter", "step"): synth.SRC_DRAFT_STEP, ("drafter", "clean"): synth.SRC_DRAFT_CLEAN,
+           ("target", "step"): synth.SRC_TARGET_STEP, ("target", "clean"): synth.SRC_TARGET_CLEAN,
+           ("target", "accepted"): synth.SRC_ACCEPT_CLEAN}
+
+    def __init__(self, sh_d, sh_t, seed):
+        self.pool = {"drafter": synth.TensorPool(sh_d, seed, n=3) if sh_d else None,
+                     "target": synth.TensorPool(sh_t, seed + 1, n=3)}
+
+    def bits(self, model, b, kind, step):
+        src = self.SRC[(model, kind)] + (step if kind == "step" else 0)
+        p = self.pool[model]
+        q = p.get(b, src, synth.Q) if kind == "step" else None
+        return q, p.get(b, src, synth.K), p.get(b, src, synth.V)
+
+    def device(self, model, b, kind, step):
+        q, k, v = self.bits(model, b, kind, step)
+        return (None if q is None else to_dev(q)), to_dev(k), to_dev(v)
+
+
+def sample_points(sh, seed, model, b, s, nheads=2, nrows=8):
+    rng = np.random.default_rng([seed, 0 if model == "drafter" else 1, b, s])
+    return np.sort(rng.choice(sh.heads, nheads, replace=False)), np.sort(rng.choice(sh.block_tokens, nrows, replace=False))
+
+
+def check_rows(got_bits, ref, what):
+    mx, mean, rel = attn_errors(got_bits, ref)
+    assert mx <= ATTN_MAX_ABS and mean <= ATTN_MEAN_ABS and rel <= 2 * ATTN_REL_RMS, (what, mx, mean, rel)
+
+
+def model_state(sh, tab_frames):
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    tab = api.sdvg_rope3d_table(sh.head_dim, tab_frames, sh.grid_h, sh.grid_w).cuda()
+    return schedule.ModelState(cache, (sh.frames, sh.grid_h, sh.grid_w), tab, tab_frames, sh.scale)
+
+
+def assert_ring_equal(cache: api.Cache, ref: O.RingCacheRef, what):
+    nb, slot_block, _ = cache.state()
+    assert nb == ref.next_block and slot_block == ref.slot_block, what
+    for s in range(ref.slots):
+        if ref.slot_block[s] < 0:
+            continue
+        gk, gv = cache.read_block(s)
+        assert np.array_equal(to_bits(gk), ref.k[s]), (what, "K", s)
+        assert np.array_equal(to_bits(gv), ref.v[s]), (what, "V", s)
+
+
+def test_config4_sweep_every_fill_level_then_eviction():
+    sh = synth.WAN_14B
+    B = 9
+    tabf = B * sh.frames
+    grid = (sh.frames, sh.grid_h, sh.grid_w)
+    prov = Provider(None, sh, 4)
+    m = model_state(sh, tabf)
+    ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ref_tab = O.rope_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w)
+    evicted = []
+    for b in range(B):
+        fo = b * sh.frames
+        for s in range(STEPS):
+            q, k, v = prov.bits("target", b, "step", s)
+            api.sdvg_rope3d_qk_commit(m.cache, to_dev(q), to_dev(k), to_dev(v), m.q_roped, None, grid, fo, m.table,
+                                      tabf, b, api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd(m.q_roped, None, None, m.cache, b, m.out, None, sh.scale, m.workspace)
+            assert api.sdvg_block_attn_status(m.workspace) == api.SDVG_OK
+            heads, rows = sample_points(sh, 4, "target", b, s)
+            qr_full_rows = O.rope_bitspec(q, grid, fo, ref_tab, tabf)[rows]
+            kr = O.rope_bitspec(k, grid, fo, ref_tab, tabf)
+            assert np.array_equal(to_bits(m.q_roped)[rows], qr_full_rows)
+            got = to_bits(m.out)
+            for h in heads:
+                q_pad = np.zeros((sh.block_tokens, sh.heads, sh.head_dim), dtype=np.uint16)
+                q_pad[rows] = qr_full_rows
+                o_ref, _ = O.block_attn_ref(q_pad, kr, v, ref, b, sh.scale, heads=[h], rows=rows)
+                check_rows(got[rows, h], o_ref[:, 0], ("sweep", b, s, h))
+        _, k, v = prov.bits("target", b, "clean", 0)
+        ev = api.sdvg_rope3d_qk_commit(m.cache, None, to_dev(k), to_dev(v), None, None, grid, fo, m.table, tabf, b,
+                                       api.SDVG_FINAL)
+        kr = O.rope_bitspec(k, grid, fo, ref_tab, tabf)
+        assert ev == ref.commit(b, kr, v, O.FINAL)
+        evicted.append(ev)
+        gk, gv = m.cache.read_block(b % sh.slots)
+        assert np.array_equal(to_bits(gk), kr) and np.array_equal(to_bits(gv), v), ("slot after commit", b)
+    assert evicted == [-1] * 7 + [0, 1]
+    assert_ring_equal(m.cache, ref, "sweep end")
+    m.cache.close()
+
+
+def run_trace(sh_d, sh_t, B, scores, tau, seed):
+    """The same trace through the oracle and through the device schedule; compares everything."""
+    tabf = B * sh_t.frames
+    prov = Provider(sh_d, sh_t, seed)
+    shapes = {"drafter": sh_d, "target": sh_t}
+
+    # ---- device
+    md, mt = model_state(sh_d, tabf), model_state(sh_t, tabf)
+    got_rows = {}
+
+    def on_attention_dev(model, b, s, q_roped, out):
+        if (b + s) % 5 == 0 or b == B - 1:
+            heads, rows = sample_points(shapes[model], seed, model, b, s)
+            got_rows[(model, b, s)] = to_bits(out[torch.from_numpy(rows).cuda()][:, torch.from_numpy(heads).cuda()])
+
+    res = schedule.run_schedule(B, STEPS, torch.from_numpy(scores).cuda(), tau, md, mt, prov.device,
+                                on_attention=on_attention_dev)
+    assert api.sdvg_block_attn_status(md.workspace) == api.SDVG_OK
+    assert api.sdvg_block_attn_status(mt.workspace) == api.SDVG_OK
+
+    # ---- oracle
+    rd = O.RingCacheRef(sh_d.slots, sh_d.heads, sh_d.block_tokens, sh_d.head_dim)
+    rt = O.RingCacheRef(sh_t.slots, sh_t.heads, sh_t.block_tokens, sh_t.head_dim)
+    tab_d = O.rope_table(sh_d.head_dim, tabf, sh_d.grid_h, sh_d.grid_w)
+    tab_t = O.rope_table(sh_t.head_dim, tabf, sh_t.grid_h, sh_t.grid_w)
+    checked = []
+
+    def on_attention_ref(model, b, s, qr, kr, v, cache):
+        if (model, b, s) not in got_rows:
+            return
+        sh = shapes[model]
+        heads, rows = sample_points(sh, seed, model, b, s)
+        o_ref, _ = O.block_attn_ref(qr, kr, v, cache, b, sh.scale, heads=list(heads), rows=rows)
+        check_rows(got_rows[(model, b, s)], o_ref, (model, b, s))
+        checked.append((model, b, s))
+
+    want = O.schedule_ref(B, STEPS, scores, tau, rd, rt, prov.bits,
+                          (sh_d.frames, sh_d.grid_h, sh_d.grid_w), (sh_t.frames, sh_t.grid_h, sh_t.grid_w),
+                          sh_t.frames, tab_d, tab_t, tabf, on_attention=on_attention_ref)
+
+    assert np.array_equal(res.accept, want.accept)
+    assert np.array_equal(res.q_min.view(np.uint32), want.q_min.view(np.uint32))
+    assert res.target_source == want.target_source
+    assert res.drafter_evicted == want.drafter_evicted and res.target_evicted == want.target_evicted
+    assert res.drafter_attn_calls == want.drafter_attn_calls == STEPS * B
+    assert res.target_attn_calls == want.target_attn_calls
+    assert sorted(checked) == sorted(got_rows)          # every sampled point was compared
+    assert_ring_equal(md.cache, rd, "drafter ring")
+    assert_ring_equal(mt.cache, rt, "target ring")
+    md.cache.close()
+    mt.cache.close()
+    return want
+
+
+def test_config5_trace_small_shapes_all_three_taus():
+    # same flow at small shapes (ragged tiles, both branches, ring wrap-around of both caches)
+    sh_d = synth.Shape("d-small", heads=3, head_dim=128, frames=3, grid_h=4, grid_w=13, slots=3)
+    sh_t = synth.Shape("t-small", heads=5, head_dim=128, frames=3, grid_h=4, grid_w=13, slots=7)
+    B = 16
+    iid = synth.normal_scores(B, 12, -0.5, 0.6, 5)
+    cal = synth.calibrated_scores(B, 12, 5)
+    for tau in (-0.9, -0.7, -0.5):
+        run_trace(sh_d, sh_t, B, iid, tau, 50)
+        want = run_trace(sh_d, sh_t, B, cal, tau, 51)
+        assert 0 < int(want.accept.sum()) < B - 1        # both branches ran
+
+
+def test_config5_trace_full_shapes_calibrated_scores():
+    # Wan-1.3B drafter + Wan-14B target, 16 blocks, scores whose block minima follow Table 1
+    B = 16
+    cal = synth.calibrated_scores(B, 12, 5)
+    want = run_trace(synth.WAN_1_3B, synth.WAN_14B, B, cal, -0.7, 52)
+    assert 0 < int(want.accept.sum()) < B - 1
+
+
+def test_config5_trace_full_shapes_iid_scores():
+    # the distribution the configuration names, N(-0.5, 0.6) per frame: (almost) every block is regenerated.
+    # The three thresholds give the same accept vector here, so the full-shape flow is run for the middle one
+    # and the routing of all three is compared on the same scores.
+    B = 16
+    iid = synth.normal_scores(B, 12, -0.5, 0.6, 5)
+    vecs = []
+    for tau in (-0.9, -0.7, -0.5):
+        a, _, _ = O.route_ref(iid.reshape(-1), None, B, 12, 0, tau)
+        acc = torch.empty(B, dtype=torch.uint8, device="cuda")
+        qm = torch.empty(B, dtype=torch.float32, device="cuda")
+        api.sdvg_route(torch.from_numpy(iid.reshape(-1)).cuda(), None, B, 12, 0, tau, acc, qm, None)
+        assert np.array_equal(acc.cpu().numpy(), a)
+        vecs.append(a.tobytes())
+    run_trace(synth.WAN_1_3B, synth.WAN_14B, B, iid, -0.7, 53)
