@@ -11,7 +11,7 @@
 // ends at the segment so that TMA zero-fills the ragged last tile; those columns are masked to
 // -inf before the row maximum.
 //
-// Every wait on an mbarrier is bounded: after kWaitLimitNs the waiting thread raises an abort flag
+// Every wait on an mbarrier is bounded: kWaitLimitNs after kernel start a waiting thread gives up
 // and writes SDVG_ERR_TIMEOUT to the status word; all roles then fall through to the common exit,
 // which releases tensor memory.
 #include <cuda.h>
@@ -62,29 +62,48 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return y;
 }
 
-struct WaitCtx {
-  volatile int* abort_flag;            // shared
-  unsigned int* status;                // global
-  uint64_t t0;                         // unused by the wait itself; kept for diagnostics
+// Every wait on an mbarrier ends at an absolute deadline taken at kernel start.
+struct Deadline {
+  uint64_t t_ns;                       // globaltimer value after which waits give up
+  unsigned int* status;                // global status word
 };
 
-// Bounded mbarrier wait: gives up kWaitLimitNs after its own first slow poll.  Returns false once
-// the CTA is aborting.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, const WaitCtx& c) {
-  uint64_t start = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 0xff) == 0xff) {
-      if (*c.abort_flag) return false;
-      const uint64_t now = globaltimer_ns();
-      if (start == 0) start = now;
-      if (now - start > kWaitLimitNs) {
-        *c.abort_flag = 1;
-        atomicExch(c.status, (unsigned)SDVG_ERR_TIMEOUT);
-        return false;
-      }
-    }
-  }
+// Slow path of the bounded wait: poll until the phase completes or the deadline passes.  Kept out
+// of line of the first attempt so that the timer read never sits on the fast path.
+__device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity, uint64_t deadline_ns,
+                                           unsigned int* status) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u64 t;\n\t"
+      "SDVG_WAIT:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra SDVG_DONE;\n\t"
+      "mov.u64 t, %%globaltimer;\n\t"
+      "setp.lt.u64 q, t, %3;\n\t"
+      "@q bra SDVG_WAIT;\n\t"
+      "SDVG_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
+      : "memory");
+  if (!ok) atomicExch(status, (unsigned)SDVG_ERR_TIMEOUT);
+  return ok != 0;
+}
+
+// Bounded mbarrier wait.  One try_wait (which itself suspends the thread for a hardware-chosen
+// time) settles almost every wait; only if it fails does the thread enter the timed poll loop.
+// Returns false (and records SDVG_ERR_TIMEOUT) once the deadline has passed.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, const Deadline& d) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return wait_bar_slow(smem_u32(bar), parity, d.t_ns, d.status);
+}
+
+// The same wait made by all 32 lanes of a warp, with a warp-uniform result.
+__device__ __forceinline__ bool wait_warp(uint64_t* bar, uint32_t parity, const Deadline& d) {
+  return __all_sync(0xffffffffu, wait_bar(bar, parity, d));
 }
 
 template <int D>
@@ -110,8 +129,6 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
   uint64_t* s_bar = full_bar + 1;
   uint64_t* o_bar = full_bar + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 3);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
   const int tid = threadIdx.x, warp = tid >> 5;
   const int qt = blockIdx.x, head = blockIdx.y;
   constexpr uint32_t kTmemCols = 256;                    // S: [0,128) (P aliases its first 64), O: [128, 128+D)
@@ -120,7 +137,6 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
     mbar_init(full_bar, 1);
     mbar_init(s_bar, 1);
     mbar_init(o_bar, 1);
-    *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&p.q_map);
   }
@@ -134,7 +150,7 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tS = tmem_base, tO = tmem_base + 128;
   const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-  WaitCtx wc{abort_flag, p.work + 1, globaltimer_ns()};
+  const Deadline wc{globaltimer_ns() + kWaitLimitNs, p.work + 1};
 
   uint32_t full_phase = 0, s_phase = 0, o_phase = 0;
   bool alive = true;
@@ -452,6 +468,11 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kWorkspaceBytes
 }  // namespace
 
 extern "C" {
+
+#ifdef SDVG_ATTN_TRACE
+// Developer build only: device buffer of [5][512][2] int64 that CTA 0 fills with (event, clock) pairs.
+int sdvg_debug_set_trace(void* p) { return (int)cudaMemcpyToSymbol(g_trace, &p, sizeof(p)); }
+#endif
 
 size_t sdvg_block_attn_workspace_bytes(void) { return kWorkspaceBytes; }
 
