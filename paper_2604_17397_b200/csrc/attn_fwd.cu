@@ -470,7 +470,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kWorkspaceBytes
 extern "C" {
 
 #ifdef SDVG_ATTN_TRACE
-// Developer build only: device buffer of [5][512][2] int64 that CTA 0 fills with (event, clock) pairs.
+// Developer build only: device buffer of [6][512][2] int64 that CTA 0 fills with (event, clock) pairs.
 int sdvg_debug_set_trace(void* p) { return (int)cudaMemcpyToSymbol(g_trace, &p, sizeof(p)); }
 #endif
 

@@ -5,7 +5,8 @@
 //
 //   warps 0-3   softmax of lane 0 (one thread per row)            \  S, P and O live in tensor memory:
 //   warps 4-7   softmax of lane 1                                  >  S0 S1 O0 O1 = 4 x 128 columns
-//   warps 8-11  correction: rescales O when a row maximum moved   /
+//   warps 8-11  helper: rescales O when a row maximum moved, and  /
+//               exponentiates the last 32 key columns of both lanes
 //   warp  12    TMA producer: Q tiles, then the K/V ring
 //   warp  13    MMA issuer: S_i = Q_i K^T, O_i += P_i V
 //   warps 14-15 idle
@@ -16,10 +17,14 @@
 // and the correction warps stay off the critical path; the final 1/l normalisation and the store
 // are done by the softmax warps themselves, which own the same TMEM lanes.
 //
-// The issuer sits on the critical path between "P is ready" and the next S, so it waits on as few
-// barriers as possible: one barrier per lane collects both the softmax threads (P stored) and the
-// correction threads (O rescaled), and the K/V stages of an iteration are checked together before
-// that.  The producer and issuer warps run their loops with all 32 lanes (warp-uniform control
+// The chain S ready -> softmax -> P ready -> PV, QK -> next S ready of one lane sets the pace, so it
+// is shortened from both ends.  A softmax thread reduces its whole row of S to the maximum, hands
+// the reference maximum to the helper thread of the same row, and exponentiates key columns 0-95;
+// the helper thread does columns 96-127 meanwhile.  P is released to the issuer in two parts
+// (columns 0-63 and 96-127 together with "O rescaled", then columns 64-95), and the issuer starts
+// the PV product on the first part while the softmax thread finishes the third quarter.  The issuer
+// is blocked while the tensor pipe's queue is full, so it looks at the K/V stages of its next step
+// right after queueing a batch of MMAs, when that costs nothing.  The producer and issuer warps run their loops with all 32 lanes (warp-uniform control
 // flow and values) and only predicate the TMA / MMA / commit instructions on one elected lane:
 // descriptors and addresses then stay in uniform registers.
 //
@@ -30,7 +35,7 @@
 #pragma once
 
 #ifdef SDVG_ATTN_TRACE
-__device__ long long* g_trace = nullptr;     // [5 roles][512 events][id, clock]
+__device__ long long* g_trace = nullptr;     // [6 roles][512 events][id, clock]
 #define SDVG_TRACE_DECL(cond)                 \
   long long* const tr_base = g_trace;         \
   const bool tr_on = (cond) && tr_base;       \
@@ -58,9 +63,9 @@ struct WsCfg {
   static constexpr int kStages = (D == 128) ? 5 : 8;                // K/V ring entries (K and V alternate)
   static constexpr int kQ = 0;                                      // two query tiles
   static constexpr int kKV = 2 * kTileBytes;
-  static constexpr int kAlpha = kKV + kStages * kTileBytes;         // float [2][128]
-  static constexpr int kBars = kAlpha + 2 * 128 * 4;
-  static constexpr int kNumBars = 16 + 2 * kStages;
+  static constexpr int kRowState = kKV + kStages * kTileBytes;      // float [2][128]: -m*c2 of a row, later the helper's l
+  static constexpr int kBars = kRowState + 2 * 128 * 4;
+  static constexpr int kNumBars = 20 + 2 * kStages;
   static constexpr int kMisc = kBars + kNumBars * 8;                // tmem slot
   static constexpr int kTotal = kMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;
@@ -115,6 +120,12 @@ struct RingPos {
       stage = 0;
       phase ^= 1;
     }
+  }
+  template <int N>
+  __device__ __forceinline__ void skip(uint32_t n) {
+    const uint32_t t = stage + n;
+    stage = t % (uint32_t)N;
+    phase ^= (t / (uint32_t)N) & 1;
   }
 };
 
@@ -180,20 +191,61 @@ __device__ __forceinline__ void exp2_poly2(uint64_t x2, float& e0, float& e1) {
 #define SDVG_ATTN_POLY_PAIRS 0
 #endif
 
+// One 32-column chunk of a row: P = 2^(c2 * S - m*c2) as bf16 pairs, returns the packed partial row sums.
+__device__ __forceinline__ void exp_chunk(const uint32_t (&s)[32], uint64_t c2x2, uint64_t negx2, uint32_t (&pk)[16],
+                                          uint64_t& sum_a, uint64_t& sum_b) {
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+    const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * k]), __uint_as_float(s[2 * k + 1])), c2x2, negx2);
+    float p0, p1;
+    if ((k & 3) < SDVG_ATTN_POLY_PAIRS) {
+      exp2_poly2(x2, p0, p1);
+    } else {
+      float x0, x1;
+      unpack2(x2, x0, x1);
+      p0 = fast_exp2(x0);
+      p1 = fast_exp2(x1);
+    }
+    if (k & 1) sum_b = add2(sum_b, pack2(p0, p1));
+    else sum_a = add2(sum_a, pack2(p0, p1));
+    __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+    pk[k] = *reinterpret_cast<uint32_t*>(&b);
+  }
+}
+
+__device__ __forceinline__ void mask_chunk(uint32_t (&s)[32], int first_col, int valid) {
+#pragma unroll
+  for (int k = 0; k < 32; ++k)
+    if (first_col + k >= valid) s[k] = 0xff800000u;      // -inf
+}
+
+__device__ __forceinline__ void max_chunk(const uint32_t (&s)[32], float (&mx)[4]) {
+#pragma unroll
+  for (int k = 0; k < 32; k += 8)
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      mx[u] = fmax3(mx[u], __uint_as_float(s[k + 2 * u]), __uint_as_float(s[k + 2 * u + 1]));
+}
+
 template <int D>
 __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_constant__ AttnParams p) {
   using C = WsCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  float* s_alpha = reinterpret_cast<float*>(smem + C::kAlpha);
+  // [2][128]: while an item runs, -m_ref * c2 of the row (softmax -> helper); at its end the helper's
+  // share of the row sum travels back through the same word
+  float* s_neg = reinterpret_cast<float*>(smem + C::kRowState);
+  float* s_lhelp = s_neg;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBars);
   uint64_t* q_full = bars;            // [2] TMA -> MMA
   uint64_t* q_empty = bars + 2;       // [2] MMA -> TMA
   uint64_t* s_full = bars + 4;        // [2] MMA -> softmax
-  uint64_t* pv_ready = bars + 6;      // [2] softmax (P stored) + correction (O rescaled) -> MMA, 256 arrivals
-  uint64_t* sm2corr = bars + 8;       // [2] softmax -> correction (128 arrivals)
-  uint64_t* o_full = bars + 10;       // [2] MMA -> correction / softmax epilogue
-  uint64_t* kv_full = bars + 16;      // [kStages]
+  uint64_t* p_lo = bars + 6;          // [2] P columns 0-63 (softmax), 96-127 + O rescaled (helper) -> MMA, 256 arrivals
+  uint64_t* p_mid = bars + 8;         // [2] P columns 64-95 stored (softmax) -> MMA, 128 arrivals
+  uint64_t* row_ready = bars + 12;    // [2] softmax -> helper: -m*c2 of the row published, 128 arrivals
+  uint64_t* o_full = bars + 14;       // [2] MMA -> helper / softmax epilogue
+  uint64_t* l_ready = bars + 16;      // [2] helper -> softmax epilogue: its share of the row sum, 128 arrivals
+  uint64_t* kv_full = bars + 20;      // [kStages]
   uint64_t* kv_empty = kv_full + C::kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kMisc);
 
@@ -204,9 +256,11 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       mbar_init(&q_full[i], 1);
       mbar_init(&q_empty[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&pv_ready[i], 256);
-      mbar_init(&sm2corr[i], 128);
+      mbar_init(&p_lo[i], 256);
+      mbar_init(&p_mid[i], 128);
+      mbar_init(&row_ready[i], 128);
       mbar_init(&o_full[i], 1);
+      mbar_init(&l_ready[i], 128);
     }
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&kv_full[s], 1);
@@ -302,29 +356,53 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, false);
       constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, true);
       const uint32_t sQ = smem_u32(smem + C::kQ), sKV = smem_u32(smem + C::kKV);
-      uint32_t q_cnt[2] = {0, 0}, pv_cnt[2] = {0, 0};
-      RingPos ring;
+      uint32_t q_cnt[2] = {0, 0};
+      uint32_t pv_par = 0;                 // bit i: phase parity of lane i's P barriers
+      RingPos ring;                        // next K/V stage to consume
       bool alive = true;
       SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
 
+      // The issue loops are deliberately not unrolled: this warp runs through its code once per key
+      // tile, between long stretches of other warps' code, and every instruction it does not have
+      // is one it does not have to fetch again.
       // S_i = Q_i K^T into TMEM columns [128 i, 128 i + 128)
       auto issue_qk = [&](int i, uint32_t st) {
-        const uint32_t a0 = sQ + i * C::kTileBytes, b0 = sKV + st * C::kTileBytes;
         const uint32_t d = tmem_base + i * 128;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * C::kPanelBytes + (kk & 3) * 32;
-          mma_ss(d, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024), kIdescQK, kk > 0);
+        uint64_t a = smem_desc_sw128(sQ + i * C::kTileBytes, 16, 1024);
+        uint64_t b = smem_desc_sw128(sKV + st * C::kTileBytes, 16, 1024);
+        uint32_t acc = 0;
+#pragma unroll 1
+        for (int h = 0; h < C::kHalves; ++h) {
+#pragma unroll 1
+          for (int k4 = 0; k4 < 4; ++k4) {
+            mma_ss(d, a + 2 * k4, b + 2 * k4, kIdescQK, acc);          // 16 bf16 = 32 B = 2 descriptor units
+            acc = 1;
+          }
+          a += C::kPanelBytes >> 4;
+          b += C::kPanelBytes >> 4;
         }
       };
-      // O_i (+)= P_i V with P_i read from the first 64 columns of S_i
-      auto issue_pv = [&](int i, uint32_t st, bool accumulate) {
-        const uint32_t b0 = sKV + st * C::kTileBytes;
+      // O_i (+)= P_i[:, 16 kk .. 16 kk + 16) V[16 kk .. 16 kk + 16, :] for kk in [k0, k1); P_i is read from
+      // the first 64 columns of S_i
+      auto issue_pv = [&](int i, uint32_t st, int k0, int k1, uint32_t acc) {
         const uint32_t d = tmem_base + 256 + i * 128, a = tmem_base + i * 128;
-#pragma unroll
-        for (int kk = 0; kk < kTileN / 16; ++kk)
-          mma_ts(d, a + kk * 8, smem_desc_sw128(b0 + kk * 2048, C::kPanelBytes, 1024), kIdescPV,
-                 (accumulate || kk > 0) ? 1u : 0u);
+        uint64_t b = smem_desc_sw128(sKV + st * C::kTileBytes, C::kPanelBytes, 1024) + (uint64_t)(k0 * (2048 >> 4));
+#pragma unroll 1
+        for (int kk = k0; kk < k1; ++kk) {
+          mma_ts(d, a + kk * 8, b, kIdescPV, acc);
+          acc = 1;
+          b += 2048 >> 4;
+        }
+      };
+      // Are the next `n` (1 or 2) stages of the ring filled?  Does not block.
+      auto stages_filled = [&](int n) {
+        RingPos r = ring;
+        bool ok = mbar_try_wait(&kv_full[r.stage], r.phase);
+        if (n > 1) {
+          r.template advance<C::kStages>();
+          ok = mbar_try_wait(&kv_full[r.stage], r.phase) && ok;
+        }
+        return __all_sync(0xffffffffu, ok);
       };
 
       for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
@@ -341,9 +419,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         if (!alive) break;
         // ---- prologue: S_i(0) ------------------------------------------------------------------
         uint32_t stK = 0;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          if (i >= nl || !alive) break;
+#pragma unroll 1
+        for (int i = 0; i < nl && alive; ++i) {
           const bool own = (i == 0) || dual;                 // this lane takes a stage of its own
           const bool last_user = dual || (i == nl - 1);
           if (own) {
@@ -359,41 +436,57 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           }
         }
         // ---- main loop -------------------------------------------------------------------------
+        bool filled = false;               // the stages of the coming step were seen filled already
         for (int j = 0; j < ntiles_k && alive; ++j) {
           const bool more = j + 1 < ntiles_k;
           uint32_t stV = 0;
           SDVG_TRACE(2, 100 + j);
-#pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            if (i >= nl || !alive) break;
+#pragma unroll 1
+          for (int i = 0; i < nl && alive; ++i) {
             const bool own = (i == 0) || dual;
             const bool last_user = dual || (i == nl - 1);
             if (own) {
-              // V_j and K_(j+1) are normally in place long before they are needed: check both first
+              // V_j and K_(j+1)
               stV = ring.stage;
               const uint32_t phV = ring.phase;
+              if (!filled) filled = stages_filled(more ? 2 : 1);
               ring.template advance<C::kStages>();
-              bool ok = mbar_try_wait(&kv_full[stV], phV);
               uint32_t phK = 0;
               if (more) {
                 stK = ring.stage;
                 phK = ring.phase;
                 ring.template advance<C::kStages>();
-                ok = mbar_try_wait(&kv_full[stK], phK) && ok;
               }
-              if (!__all_sync(0xffffffffu, ok)) {
+              if (!filled) {
                 if (!(alive = wait_warp(&kv_full[stV], phV, dl))) break;
                 if (more && !(alive = wait_warp(&kv_full[stK], phK, dl))) break;
               }
+              filled = false;
             }
             SDVG_TRACE(2, 1000 + i * 1000 + j);
-            // P_i(j) stored and O_i rescaled (for j = 0: O_i read out by the previous epilogue)
-            if (!(alive = wait_warp(&pv_ready[i], pv_cnt[i] & 1, dl))) break;
-            ++pv_cnt[i];
+            const uint32_t par = (pv_par >> i) & 1;
+            pv_par ^= 1u << i;
+            // P_i(j) columns 0-63 and 96-127 stored, O_i rescaled (for j = 0: O_i was read out by the
+            // epilogue of the previous item before its softmax threads arrived here)
+            if (!(alive = wait_warp(&p_lo[i], par, dl))) break;
             SDVG_TRACE(2, 3000 + i * 1000 + j);
             tc_fence_after();
             if (leader) {
-              issue_pv(i, stV, j > 0);
+              issue_pv(i, stV, 6, 8, j > 0 ? 1u : 0u);
+              issue_pv(i, stV, 0, 4, 1u);
+            }
+            // six MMAs are queued: a good moment to look at the stages of the next step that takes any
+            {
+              const bool next_in_this_j = dual && (i + 1 < nl);
+              const bool next_more = next_in_this_j ? more : (j + 2 < ntiles_k);
+              if ((next_in_this_j || (last_user && more)) && (dual || i == nl - 1))
+                filled = stages_filled(next_more ? 2 : 1);
+            }
+            if (!(alive = wait_warp(&p_mid[i], par, dl))) break;
+            SDVG_TRACE(2, 5000 + i * 1000 + j);
+            tc_fence_after();
+            if (leader) {
+              issue_pv(i, stV, 4, 6, 1u);
               mma_commit(&o_full[i]);
               if (last_user) mma_commit(&kv_empty[stV]);
               if (more) {
@@ -410,33 +503,41 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       }
     }
   } else if (warp >= 8) {
-    // ================= correction warps ========================================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    // ================= helper warps =============================================================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
     const int row = tid - 256;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS[2] = {tmem_base + lane_off, tmem_base + 128 + lane_off};
     const uint32_t tO[2] = {tmem_base + 256 + lane_off, tmem_base + 384 + lane_off};
-    uint32_t a_cnt[2] = {0, 0}, pv_cnt[2] = {0, 0};
+    const float c2 = p.scale_log2e;
+    const uint64_t c2x2 = pack2(c2, c2);
+    uint32_t cnt[2] = {0, 0};            // (item, key tile) steps done per lane = phase index of its barriers
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && tid == 256)
     for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
       WsItem it;
       sched.get(v, it);
-      for (int j = 0; j < ntiles_k && alive; ++j) {
+      float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
+      int j = 0;
+      for (int seg = 0; seg < p.nseg && alive; ++seg) {
+        const int len = p.seg_len[seg];
+        const int nt = (len + kTileN - 1) / kTileN;
+        for (int kt = 0; kt < nt && alive; ++kt, ++j) {
+          const int valid = min(kTileN, len - kt * kTileN);
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          if (i >= it.lanes || !alive) break;
-          if (j == 0) {
-            // Nothing to rescale yet.  The arrival below must not fall into the previous phase of
-            // pv_ready (the last key tile of the previous item), so that phase has to be over.
-            if (pv_cnt[i] > 0 && !(alive = wait_bar(&pv_ready[i], (pv_cnt[i] - 1) & 1, dl))) break;
-          } else {
-            if (!(alive = wait_bar(&sm2corr[i], a_cnt[i] & 1, dl))) break;
-            ++a_cnt[i];
-            const float alpha = s_alpha[i * 128 + row];
+          for (int i = 0; i < 2; ++i) {
+            if (i >= it.lanes || !alive) break;
+            const uint32_t par = cnt[i] & 1;
+            if (!(alive = wait_bar(&row_ready[i], par, dl))) break;
+            const float neg = s_neg[i * 128 + row];
+            // the row's reference maximum moved iff -m*c2 changed; both sides derive the factor the same way
+            const bool moved = (j > 0) && (neg != neg_prev[i]);
+            const float alpha = moved ? fast_exp2(__fsub_rn(neg, neg_prev[i])) : 1.f;
+            neg_prev[i] = neg;
             SDVG_TRACE(3, 1000 * i + j);
-            if (__any_sync(0xffffffffu, alpha != 1.f)) {
-              // PV_i(j-1) is MMA number pv_cnt[i] - 1 on o_full[i]
-              if (!(alive = wait_bar(&o_full[i], (pv_cnt[i] - 1) & 1, dl))) break;
+            if (__any_sync(0xffffffffu, moved)) {
+              // PV_i(j-1) is commit number cnt[i] - 1 on o_full[i]
+              if (!(alive = wait_bar(&o_full[i], (cnt[i] - 1) & 1, dl))) break;
               tc_fence_after();
 #pragma unroll
               for (int c = 0; c < D / 32; ++c) {
@@ -449,17 +550,44 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
               }
               tmem_wait_st();
               tc_fence_before();
+              l_part[i] *= alpha;
             }
+            SDVG_TRACE(3, 20000 + 1000 * i + j);
+            // ---- this row's share of P: key columns 96-127 -------------------------------------
+            tc_fence_after();
+            uint32_t s3[32], pk[16];
+            tmem_ld32(tS[i] + 96, s3);
+            tmem_wait_ld();
+            if (valid < kTileN) mask_chunk(s3, 96, valid);
+            uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
+            exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
+            tmem_st16(tS[i] + 48, pk);
+            {
+              float a0, a1, b0, b1;
+              unpack2(sum_a, a0, a1);
+              unpack2(sum_b, b0, b1);
+              l_part[i] += (a0 + a1) + (b0 + b1);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&p_lo[i]);
+            SDVG_TRACE(3, 30000 + 1000 * i + j);
+            ++cnt[i];
           }
-          SDVG_TRACE(3, 20000 + 1000 * i + j);
-          mbar_arrive(&pv_ready[i]);
-          ++pv_cnt[i];
         }
+      }
+      if (!alive) break;
+      // hand the partial row sums to the softmax threads that normalise and store the rows
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (i >= it.lanes) break;
+        s_lhelp[i * 128 + row] = l_part[i];
+        mbar_arrive(&l_ready[i]);
       }
     }
   } else {
     // ================= softmax warps ===========================================================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 176;");
     const int i = warp >> 2;                       // lane (query tile) of this warpgroup
     const int row = tid & 127;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -467,14 +595,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     const uint32_t tO = tmem_base + 256 + i * 128 + lane_off;
     const float c2 = p.scale_log2e;
     const uint64_t c2x2 = pack2(c2, c2);
-    uint32_t s_cnt = 0, pv_cnt = 0;
+    uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0;
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0)
     for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
       WsItem it;
       sched.get(v, it);
       if (it.lanes <= i) continue;
-      float m_ref = -INFINITY, l_run = 0.f;
+      float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2
       int j = 0;
       for (int seg = 0; seg < p.nseg && alive; ++seg) {
         const int len = p.seg_len[seg];
@@ -486,104 +614,77 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           SDVG_TRACE(i, 1000 + j);
           ++s_cnt;
           tc_fence_after();
-          // ---- row maximum; the second half of S streams in while the first is reduced -----
-          uint32_t s[4][32];
-          tmem_ld32(tS, s[0]);
-          tmem_ld32(tS + 32, s[1]);
-          tmem_wait_ld();
-          tmem_ld32(tS + 64, s[2]);
-          tmem_ld32(tS + 96, s[3]);
+          // ---- row maximum over all 128 columns; the second half streams in while the first is reduced
+          uint32_t s[3][32];
           float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          if (valid < kTileN) {
-#pragma unroll
-            for (int c = 0; c < 2; ++c)
-#pragma unroll
-              for (int k = 0; k < 32; ++k)
-                if (c * 32 + k >= valid) s[c][k] = 0xff800000u;      // -inf
-          }
-#pragma unroll
-          for (int c = 0; c < 2; ++c)
-#pragma unroll
-            for (int k = 0; k < 32; k += 8) {
-#pragma unroll
-              for (int u = 0; u < 4; ++u)
-                mx[u] = fmax3(mx[u], __uint_as_float(s[c][k + 2 * u]), __uint_as_float(s[c][k + 2 * u + 1]));
+          {
+            uint32_t s3[32];
+            tmem_ld32(tS + 96, s3);
+            tmem_ld32(tS, s[0]);
+            tmem_wait_ld();
+            tmem_ld32(tS + 32, s[1]);
+            tmem_ld32(tS + 64, s[2]);
+            if (valid < kTileN) {
+              mask_chunk(s3, 96, valid);
+              mask_chunk(s[0], 0, valid);
             }
+            max_chunk(s3, mx);
+            max_chunk(s[0], mx);
+          }
           tmem_wait_ld();
           SDVG_TRACE(i, 2000 + j);
           if (valid < kTileN) {
-#pragma unroll
-            for (int c = 2; c < 4; ++c)
-#pragma unroll
-              for (int k = 0; k < 32; ++k)
-                if (c * 32 + k >= valid) s[c][k] = 0xff800000u;
+            mask_chunk(s[1], 32, valid);
+            mask_chunk(s[2], 64, valid);
           }
-#pragma unroll
-          for (int c = 2; c < 4; ++c)
-#pragma unroll
-            for (int k = 0; k < 32; k += 8) {
-#pragma unroll
-              for (int u = 0; u < 4; ++u)
-                mx[u] = fmax3(mx[u], __uint_as_float(s[c][k + 2 * u]), __uint_as_float(s[c][k + 2 * u + 1]));
-            }
+          max_chunk(s[1], mx);
+          max_chunk(s[2], mx);
           const float mxa = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
           if (j == 0) {
             m_ref = mxa;
-          } else {
-            float alpha = 1.f;
-            if ((mxa - m_ref) * c2 > 8.f) {
-              alpha = fast_exp2((m_ref - mxa) * c2);
-              m_ref = mxa;
-              l_run *= alpha;
-            }
-            s_alpha[i * 128 + row] = alpha;
-            mbar_arrive(&sm2corr[i]);
+            neg = __fmul_rn(-mxa, c2);
+          } else if ((mxa - m_ref) * c2 > 8.f) {
+            const float neg_new = __fmul_rn(-mxa, c2);
+            l_run *= fast_exp2(__fsub_rn(neg_new, neg));      // the helper derives the same factor from the same two values
+            m_ref = mxa;
+            neg = neg_new;
           }
+          s_neg[i * 128 + row] = neg;
+          mbar_arrive(&row_ready[i]);
           SDVG_TRACE(i, 3000 + j);
-          // ---- P = 2^(c2 * (S - m_ref)), bf16, written back over S ---------------------------
-          const float neg = -m_ref * c2;
+          // ---- P = 2^(c2 * (S - m_ref)), bf16, written back over S: columns 0-63, then 64-95 ------
           const uint64_t negx2 = pack2(neg, neg);
           uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int k = 0; k < 16; ++k) {
-              const uint64_t x2 =
-                  fma2(pack2(__uint_as_float(s[c][2 * k]), __uint_as_float(s[c][2 * k + 1])), c2x2, negx2);
-              float p0, p1;
-              if ((k & 3) < SDVG_ATTN_POLY_PAIRS) {
-                exp2_poly2(x2, p0, p1);
-              } else {
-                float x0, x1;
-                unpack2(x2, x0, x1);
-                p0 = fast_exp2(x0);
-                p1 = fast_exp2(x1);
-              }
-              if (k & 1) sum_b = add2(sum_b, pack2(p0, p1));
-              else sum_a = add2(sum_a, pack2(p0, p1));
-              __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-              pk[k] = *reinterpret_cast<uint32_t*>(&b);
-            }
-            tmem_st16(tS + c * 16, pk);
-          }
+          uint32_t pk[16];
+          exp_chunk(s[0], c2x2, negx2, pk, sum_a, sum_b);
+          tmem_st16(tS, pk);
+          exp_chunk(s[1], c2x2, negx2, pk, sum_a, sum_b);
+          tmem_st16(tS + 16, pk);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&p_lo[i]);
+          SDVG_TRACE(i, 4000 + j);
+          exp_chunk(s[2], c2x2, negx2, pk, sum_a, sum_b);
+          tmem_st16(tS + 32, pk);
           {
             float a0, a1, b0, b1;
             unpack2(sum_a, a0, a1);
             unpack2(sum_b, b0, b1);
             l_run += (a0 + a1) + (b0 + b1);
           }
-          SDVG_TRACE(i, 4000 + j);
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(&pv_ready[i]);
+          mbar_arrive(&p_mid[i]);
           SDVG_TRACE(i, 5000 + j);
         }
       }
       if (!alive) break;
-      // ---- epilogue: wait for the last PV of this item, normalise, store ------------------
-      // (the next item's first arrival on pv_ready comes after these TMEM reads, which is what
-      // lets the issuer overwrite O_i then)
+      // ---- epilogue: add the helper's share of the row sum, wait for the last PV, normalise, store
+      // (the next item's first arrival on p_lo comes after these TMEM reads, which is what lets the
+      // issuer overwrite O_i then)
+      if (!(alive = wait_bar(&l_ready[i], item_cnt & 1, dl))) break;
+      ++item_cnt;
+      l_run += s_lhelp[i * 128 + row];
       pv_cnt += ntiles_k;
       if (!(alive = wait_bar(&o_full[i], (pv_cnt - 1) & 1, dl))) break;
       tc_fence_after();
@@ -612,7 +713,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       }
       tc_fence_before();
       if (p.lse && grow < p.tokens)
-        p.lse[(size_t)head * p.tokens + grow] = (m_ref * c2) * 0.6931471805599453f + logf(l_run);
+        p.lse[(size_t)head * p.tokens + grow] = -neg * 0.6931471805599453f + logf(l_run);
     }
   }
 
