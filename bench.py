@@ -29,6 +29,9 @@ if ROOT not in sys.path:
 METRIC = "block-attn TFLOP/s per denoise step @14B shape (% bf16 peak); KV-commit GB/s"
 ROUTE_BLOCKS = 1003 * 9          # the paper's evaluation volume: 1003 videos x 9 blocks (Sec. 4.1)
 ROUTE_FRAMES = 12
+# DRAM bytes (read + write) of ONE attention launch, from an ncu capture of the kernel as it stands
+# (profiles/attn_fwd_ws_14b_dram.md); None for workloads that were not captured.
+ATTN_DRAM_BYTES_PER_LAUNCH = {"14b": 1.3756e9}
 CPU_SAMPLE_HEADS = 12           # heads of one step the CPU oracle is timed on (about 10-20 s of host work)
 
 
@@ -337,7 +340,9 @@ def run_ours(args):
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": attn_tflops / pk["bf16_tflops"],
                      "frac_of_sustained_peak": attn_tflops / pk["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": attn_tflops / 2250.0, "peak_source": pk["source"],
-                     "ms_per_launch": attn_ms, "traffic": None},
+                     "ms_per_launch": attn_ms, "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get(args.workload),
+                     "traffic_unit": "DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
+                     "algorithmic_hbm_bytes": (2 * sh.block_tokens + 2 * st.lk) * sh.heads * sh.head_dim * 2},
         "hbm_kernels": {
             "peak_gbs": pk["hbm_gbs"],
             "rope_stage": {"ms": t_rope, "gbs": hb["rope_stage"] / t_rope / 1e6,
