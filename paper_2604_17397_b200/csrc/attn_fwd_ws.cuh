@@ -24,8 +24,8 @@
 // (columns 0-63 and 96-127 together with "O rescaled", then columns 64-95), and the issuer starts
 // the PV product on the first part while the softmax thread finishes the third quarter.  The issuer
 // is blocked while the tensor pipe's queue is full, so it looks at the K/V stages of its next step
-// right after queueing a batch of MMAs, when that costs nothing.  The producer and issuer warps run their loops with all 32 lanes (warp-uniform control
-// flow and values) and only predicate the TMA / MMA / commit instructions on one elected lane:
+// right after queueing a batch of MMAs, when that costs nothing.  The producer and issuer warps
+// run their loops with all 32 lanes (warp-uniform control flow and values) and only predicate the TMA / MMA / commit instructions on one elected lane:
 // descriptors and addresses then stay in uniform registers.
 //
 // The exponentials are the co-limiter of this kernel: a 128 x 128 tile needs 16384 of them and the
@@ -213,12 +213,6 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&s)[32], uint64_t c2x2
   }
 }
 
-__device__ __forceinline__ void mask_chunk(uint32_t (&s)[32], int first_col, int valid) {
-#pragma unroll
-  for (int k = 0; k < 32; ++k)
-    if (first_col + k >= valid) s[k] = 0xff800000u;      // -inf
-}
-
 __device__ __forceinline__ void max_chunk(const uint32_t (&s)[32], float (&mx)[4]) {
 #pragma unroll
   for (int k = 0; k < 32; k += 8)
@@ -320,6 +314,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         ++kv_issued;
       };
 
+      #pragma unroll 1
       for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
         WsItem it;
         sched.get(v, it);
@@ -338,6 +333,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         // K/V tiles in the order the issuer consumes them
         const int streams = it.dual ? it.lanes : 1;
         for (int s = 0; s < streams && alive; ++s) load_kv(false, it.head[s], 0);
+        #pragma unroll 1
         for (int j = 0; j < ntiles_k && alive; ++j)
           for (int s = 0; s < streams && alive; ++s) {
             load_kv(true, it.head[s], j);
@@ -405,6 +401,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         return __all_sync(0xffffffffu, ok);
       };
 
+      #pragma unroll 1
       for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
         WsItem it;
         sched.get(v, it);
@@ -437,6 +434,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         }
         // ---- main loop -------------------------------------------------------------------------
         bool filled = false;               // the stages of the coming step were seen filled already
+        #pragma unroll 1
         for (int j = 0; j < ntiles_k && alive; ++j) {
           const bool more = j + 1 < ntiles_k;
           uint32_t stV = 0;
@@ -514,16 +512,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     uint32_t cnt[2] = {0, 0};            // (item, key tile) steps done per lane = phase index of its barriers
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && tid == 256)
+    #pragma unroll 1
     for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
       WsItem it;
       sched.get(v, it);
       float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
-      int j = 0;
-      for (int seg = 0; seg < p.nseg && alive; ++seg) {
-        const int len = p.seg_len[seg];
-        const int nt = (len + kTileN - 1) / kTileN;
-        for (int kt = 0; kt < nt && alive; ++kt, ++j) {
-          const int valid = min(kTileN, len - kt * kTileN);
+      #pragma unroll 1
+      for (int j = 0; j < ntiles_k && alive; ++j) {
+        {
 #pragma unroll
           for (int i = 0; i < 2; ++i) {
             if (i >= it.lanes || !alive) break;
@@ -539,8 +535,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
               // PV_i(j-1) is commit number cnt[i] - 1 on o_full[i]
               if (!(alive = wait_bar(&o_full[i], (cnt[i] - 1) & 1, dl))) break;
               tc_fence_after();
-#pragma unroll
-              for (int c = 0; c < D / 32; ++c) {
+#pragma unroll 1
+              for (int c = 0; c < D / 32; ++c) {          // rare path: keep its code small
                 uint32_t o[32];
                 tmem_ld32(tO[i] + c * 32, o);
                 tmem_wait_ld();
@@ -558,7 +554,6 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             uint32_t s3[32], pk[16];
             tmem_ld32(tS[i] + 96, s3);
             tmem_wait_ld();
-            if (valid < kTileN) mask_chunk(s3, 96, valid);
             uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
             exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
             tmem_st16(tS[i] + 48, pk);
@@ -598,15 +593,18 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0;
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0)
+    #pragma unroll 1
     for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
       WsItem it;
       sched.get(v, it);
       if (it.lanes <= i) continue;
       float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2
       int j = 0;
+      #pragma unroll 1
       for (int seg = 0; seg < p.nseg && alive; ++seg) {
         const int len = p.seg_len[seg];
         const int nt = (len + kTileN - 1) / kTileN;
+        #pragma unroll 1
         for (int kt = 0; kt < nt && alive; ++kt, ++j) {
           const int valid = min(kTileN, len - kt * kTileN);
           SDVG_TRACE(i, 0 + j);
@@ -614,6 +612,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           SDVG_TRACE(i, 1000 + j);
           ++s_cnt;
           tc_fence_after();
+          if (valid < kTileN) {
+            // Ragged last tile of a key segment (TMA zero-filled the missing keys): overwrite their
+            // columns of S with -inf in tensor memory, for this thread and for the helper thread of the
+            // row, which reads its columns after row_ready.  Rare, so a plain column-by-column loop.
+#pragma unroll 1
+            for (int c = valid; c < kTileN; ++c) tmem_st1(tS + c, 0xff800000u);
+            tmem_wait_st();
+          }
           // ---- row maximum over all 128 columns; the second half streams in while the first is reduced
           uint32_t s[3][32];
           float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -624,19 +630,11 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             tmem_wait_ld();
             tmem_ld32(tS + 32, s[1]);
             tmem_ld32(tS + 64, s[2]);
-            if (valid < kTileN) {
-              mask_chunk(s3, 96, valid);
-              mask_chunk(s[0], 0, valid);
-            }
             max_chunk(s3, mx);
             max_chunk(s[0], mx);
           }
           tmem_wait_ld();
           SDVG_TRACE(i, 2000 + j);
-          if (valid < kTileN) {
-            mask_chunk(s[1], 32, valid);
-            mask_chunk(s[2], 64, valid);
-          }
           max_chunk(s[1], mx);
           max_chunk(s[2], mx);
           const float mxa = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
@@ -691,8 +689,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       const int grow = it.tile[i] * kTileM + row;
       const int head = it.head[i];
       const float inv = 1.f / l_run;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {                  // once per item: keep its code small
         uint32_t o[32];
         tmem_ld32(tO + c * 32, o);
         tmem_wait_ld();
