@@ -197,29 +197,70 @@ class Step:
         self.attn_events = []
         self.lk = sh.slots * sh.block_tokens
 
-    def step(self, time_attention: bool = False):
+    def step(self, time_attention: bool = False, io=None):
+        """One step on the current stream; `io` = (q, k, v, scores, out, accept) device tensors to use."""
         api, sh, b = self.api, self.sh, self.block
-        api.sdvg_rope3d_qk_commit(self.cache, self.q, self.k, self.v, self.q_r, self.k_r, self.grid, b * sh.frames,
+        q, k, v, scores, out, accept = io if io is not None else (self.q, self.k, self.v, self.scores, self.out,
+                                                                  self.accept)
+        api.sdvg_rope3d_qk_commit(self.cache, q, k, v, self.q_r, self.k_r, self.grid, b * sh.frames,
                                   self.tab, self.tabf, b, api.SDVG_STAGE)
         if time_attention:
             e0, e1 = self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
             e0.record()
-        api.sdvg_block_attn_fwd(self.q_r, None, None, self.cache, b, self.out, None, sh.scale, self.ws)
+        api.sdvg_block_attn_fwd(self.q_r, None, None, self.cache, b, out, None, sh.scale, self.ws)
         if time_attention:
             e1.record()
             self.attn_events.append((e0, e1))
-        api.sdvg_kv_commit(self.cache, self.k_r, self.v, b, api.SDVG_FINAL)
-        api.sdvg_route(self.scores, None, ROUTE_BLOCKS, ROUTE_FRAMES, 0, -0.7, self.accept, self.qmin, None)
+        api.sdvg_kv_commit(self.cache, self.k_r, v, b, api.SDVG_FINAL)
+        api.sdvg_route(scores, None, ROUTE_BLOCKS, ROUTE_FRAMES, 0, -0.7, accept, self.qmin, None)
         self.block += 1
     LAUNCHES_PER_STEP = 4          # rope+stage, attention, commit, route
 
+    def e2e_setup(self):
+        """Double-buffered inputs and outputs plus one stream each for upload, compute and download, so that
+        the copies of neighbouring steps overlap the kernels (every step still uploads its own q, k, v and
+        scores from pinned host memory and downloads its own output and accept flags)."""
+        torch = self.torch
+        self.io = []
+        for _ in range(2):
+            self.io.append((torch.empty_like(self.q), torch.empty_like(self.k), torch.empty_like(self.v),
+                            torch.empty_like(self.scores), torch.empty_like(self.out), torch.empty_like(self.accept)))
+        self.out_hosts = [torch.empty_like(self.out_host).pin_memory() for _ in range(2)]
+        self.accept_hosts = [torch.empty_like(self.accept_host).pin_memory() for _ in range(2)]
+        self.s_in, self.s_comp, self.s_out = (torch.cuda.Stream() for _ in range(3))
+        self.ev_in = [torch.cuda.Event() for _ in range(2)]
+        self.ev_comp = [torch.cuda.Event() for _ in range(2)]
+        self.ev_out = [torch.cuda.Event() for _ in range(2)]
+        self.e2e_n = 0
+
     def step_e2e(self):
-        for d, h in zip((self.q, self.k, self.v), self.host):
-            d.copy_(h, non_blocking=True)
-        self.scores.copy_(self.scores_host, non_blocking=True)
-        self.step()
-        self.out_host.copy_(self.out, non_blocking=True)
-        self.accept_host.copy_(self.accept, non_blocking=True)
+        torch = self.torch
+        b = self.e2e_n % 2
+        q, k, v, scores, out, accept = self.io[b]
+        with torch.cuda.stream(self.s_in):
+            self.s_in.wait_event(self.ev_comp[b])           # the step that last read this input set is done
+            for d, h in zip((q, k, v), self.host):
+                d.copy_(h, non_blocking=True)
+            scores.copy_(self.scores_host, non_blocking=True)
+            self.ev_in[b].record()
+        with torch.cuda.stream(self.s_comp):
+            self.s_comp.wait_event(self.ev_in[b])
+            self.s_comp.wait_event(self.ev_out[b])          # this output set has been downloaded
+            self.step(io=self.io[b])
+            self.ev_comp[b].record()
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_comp[b])
+            self.out_hosts[b].copy_(out, non_blocking=True)
+            self.accept_hosts[b].copy_(accept, non_blocking=True)
+            self.ev_out[b].record()
+        self.e2e_n += 1
+
+    def e2e_join(self):
+        """Make the current stream wait for everything the three streams have been given."""
+        cur = self.torch.cuda.current_stream()
+        for evs in (self.ev_in, self.ev_comp, self.ev_out):
+            for e in evs:
+                cur.wait_event(e)
 
     def e2e_bytes(self):
         h2d = sum(h.numel() * h.element_size() for h in self.host) + self.scores_host.numel() * 4
@@ -298,15 +339,19 @@ def run_ours(args):
     t_route = time_call(lambda: api.sdvg_route(st.scores, None, ROUTE_BLOCKS, ROUTE_FRAMES, 0, -0.7, st.accept,
                                                st.qmin, None))
 
-    # end to end through the same calls with host buffers: H2D of q,k,v,scores and D2H of out, accept per step
-    for _ in range(2):
+    # end to end through the same calls with host buffers: H2D of q,k,v,scores and D2H of out, accept per step,
+    # copies of neighbouring steps overlapped with the kernels on separate streams
+    st.e2e_setup()
+    for _ in range(3):
         st.step_e2e()
+    st.e2e_join()
     torch.cuda.synchronize()
     dist_util.barrier(world)
     n_e2e = max(3, args.steps // 2)
     e0.record()
     for _ in range(n_e2e):
         st.step_e2e()
+    st.e2e_join()
     e1.record()
     torch.cuda.synchronize()
     ms_e2e = dist_util.max_over_ranks(e0.elapsed_time(e1), world, device) / n_e2e
@@ -334,7 +379,8 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks,
         "e2e": {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "overlap": "upload, kernels and download of neighbouring steps on three streams, double-buffered"},
         "gpu_launches": Step.LAUNCHES_PER_STEP * args.steps,
         "roofline": {"bound": "tensor", "kernel": "sdvg_block_attn_fwd", "achieved": attn_tflops,
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": attn_tflops / pk["bf16_tflops"],
