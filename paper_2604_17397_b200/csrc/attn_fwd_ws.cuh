@@ -390,13 +390,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           b += 2048 >> 4;
         }
       };
-      // Are the next `n` (1 or 2) stages of the ring filled?  Does not block.
+      // Are the next `n` (1 or 2) stages of the ring filled?  Does not block (test_wait, not try_wait,
+      // which may suspend the thread for microseconds when the answer is no).
       auto stages_filled = [&](int n) {
         RingPos r = ring;
-        bool ok = mbar_try_wait(&kv_full[r.stage], r.phase);
+        bool ok = mbar_test_wait(&kv_full[r.stage], r.phase);
         if (n > 1) {
           r.template advance<C::kStages>();
-          ok = mbar_try_wait(&kv_full[r.stage], r.phase) && ok;
+          ok = mbar_test_wait(&kv_full[r.stage], r.phase) && ok;
         }
         return __all_sync(0xffffffffu, ok);
       };

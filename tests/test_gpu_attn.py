@@ -73,6 +73,15 @@ def test_d64_multi_tile():
     run_sequence(sh, 6, 42, True)
 
 
+@pytest.mark.parametrize("heads,dim", [(3, 128), (1, 64), (5, 64)])
+def test_odd_tile_count_with_odd_head_count(heads, dim):
+    # 300 tokens = 3 query tiles per head: the third tiles of two heads share a work item, and with an odd
+    # number of heads the last such item has a single lane
+    sh = synth.Shape("odd-odd", heads=heads, head_dim=dim, frames=1, grid_h=12, grid_w=25, slots=3)
+    run_sequence(sh, 4, 45 + heads, True)
+    run_sequence(sh, 2, 46 + heads, False)
+
+
 def test_peaky_logits_keep_the_absolute_tolerance():
     # q scaled x4: softmax concentrates on few keys and outputs are O(1)
     sh = synth.Shape("peaky", heads=2, head_dim=128, frames=1, grid_h=12, grid_w=25, slots=3)
