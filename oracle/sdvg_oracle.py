@@ -345,6 +345,78 @@ def route_ref(scores: np.ndarray, frame_offsets, num_blocks: int, frames_per_blo
     return accept, q_min, argmin
 
 
+AGG_MIN = 0      # Eq. (1): worst frame
+AGG_MEAN = 1     # Table 2 "Avg-frame scoring": mean of the frame scores
+SIGNAL_REWARD = 0   # accept iff aggregate >= tau
+SIGNAL_RANDOM = 1   # Table 2 "random routing": accept iff a uniform draw < p, the scores are ignored
+
+
+def route_policy_ref(scores, frame_offsets, num_blocks: int, frames_per_block: int, first_block_index: int,
+                     tau: float, agg: int = AGG_MIN, signal: int = SIGNAL_REWARD, force_first: bool = True,
+                     blocks_per_video: int = 0, uniforms=None, accept_prob: float = 0.0):
+    """Routing policy with the variants of the ablation (Sec. 4.3, Table 2).
+
+    Aggregate per block: the worst frame (AGG_MIN, same rules as ``route_ref``) or the fp32 mean
+    (AGG_MEAN): the frames are added left to right, every partial sum rounded to fp32, and the sum is
+    divided by float32(F) with one more rounding.  Decision: aggregate >= tau (SIGNAL_REWARD), or
+    uniforms[b] < float32(accept_prob) with the scores ignored (SIGNAL_RANDOM; the draws are an input).
+    ``force_first`` rejects the first block of every video whatever the signal says: global block
+    g = first_block_index + b is a first block iff g == 0 (blocks_per_video == 0, one endless stream) or
+    g % blocks_per_video == 0.  "Force-reject + random" and plain "Random routing" of Table 2 differ
+    only in that flag.  Returns (accept u8[B], aggregate f32[B], argmin i32[B]; argmin is -1 for AGG_MEAN).
+    """
+    s = np.asarray(scores, dtype=np.float32).reshape(-1)
+    tau32 = np.float32(tau)
+    p32 = np.float32(accept_prob)
+    accept = np.zeros(num_blocks, dtype=np.uint8)
+    aggv = np.zeros(num_blocks, dtype=np.float32)
+    argmin = np.full(num_blocks, -1, dtype=np.int32)
+    for b in range(num_blocks):
+        if frame_offsets is None:
+            lo, hi = b * frames_per_block, (b + 1) * frames_per_block
+        else:
+            lo, hi = int(frame_offsets[b]), int(frame_offsets[b + 1])
+        if hi <= lo:
+            raise ValueError("a block needs at least one frame")
+        if agg == AGG_MIN:
+            m, idx = s[lo], 0
+            for i in range(lo + 1, hi):
+                if np.isnan(m):
+                    break
+                x = s[i]
+                if np.isnan(x) or x < m:
+                    m, idx = x, i - lo
+            argmin[b] = idx
+        elif agg == AGG_MEAN:
+            acc = np.float32(s[lo])
+            with np.errstate(invalid="ignore", over="ignore"):
+                for i in range(lo + 1, hi):
+                    acc = np.float32(acc + s[i])
+                m = np.float32(acc / np.float32(hi - lo))
+        else:
+            raise ValueError("unknown aggregation")
+        aggv[b] = m
+        g = first_block_index + b
+        first = (g == 0) if blocks_per_video == 0 else (g % blocks_per_video == 0)
+        if signal == SIGNAL_REWARD:
+            ok = (not np.isnan(m)) and m >= tau32
+        elif signal == SIGNAL_RANDOM:
+            ok = bool(np.float32(uniforms[b]) < p32)
+        else:
+            raise ValueError("unknown signal")
+        accept[b] = 1 if (ok and not (force_first and first)) else 0
+    return accept, aggv, argmin
+
+
+def accept_stats_ref(accept, first_block_index: int = 0, blocks_per_video: int = 0):
+    """(accepted, routable) block counts, the first block of every video left out of both
+    (accept-rate convention of Tables 1 and 2: "excludes block 0 (always force-rejected)")."""
+    a = np.asarray(accept).astype(np.int64)
+    g = np.arange(a.size, dtype=np.int64) + first_block_index
+    first = (g == 0) if blocks_per_video == 0 else (g % blocks_per_video == 0)
+    return int(a[~first].sum()), int((~first).sum())
+
+
 def accept_rate(accept: np.ndarray, first_block_index: int = 0) -> float:
     """Accept rate with block 0 left out of the count (convention of Tables 1 and 2)."""
     a = np.asarray(accept).astype(np.int64)

@@ -374,6 +374,77 @@ def test_calibrated_scores_follow_table1_accept_rates():
         assert O.accept_rate(a) == pytest.approx(float(rate), abs=0.01)
 
 
+def _policy_row(row):
+    blk, bpv, tau, agg, sig, force, u, p, scores, accept, aggv = row
+    s = np.array([float(t) for t in scores.split()], dtype=np.float32)
+    kw = dict(agg=O.AGG_MEAN if agg == "mean" else O.AGG_MIN,
+              signal=O.SIGNAL_RANDOM if sig == "random" else O.SIGNAL_REWARD, force_first=bool(int(force)),
+              blocks_per_video=int(bpv), uniforms=np.array([float(u)], dtype=np.float32), accept_prob=float(p))
+    return s, int(blk), float(tau), kw, int(accept), np.float32(float(aggv))
+
+
+def test_route_policy_hand_worked_cases():
+    for row in read_golden_rows("route_policy_cases.txt"):
+        s, blk, tau, kw, accept, aggv = _policy_row(row)
+        a, v, _ = O.route_policy_ref(s, None, 1, s.size, blk, tau, **kw)
+        assert int(a[0]) == accept, row
+        assert (np.isnan(aggv) and np.isnan(v[0])) or v[0] == aggv, row
+
+
+def test_route_policy_reduces_to_the_default_router():
+    s = synth.normal_scores(40, 12, -0.5, 0.6, 8)
+    for first in (0, 3):
+        a, q, i = O.route_ref(s.reshape(-1), None, 40, 12, first, -0.7)
+        a2, q2, i2 = O.route_policy_ref(s.reshape(-1), None, 40, 12, first, -0.7)
+        assert np.array_equal(a, a2) and np.array_equal(q.view(np.uint32), q2.view(np.uint32)) and np.array_equal(i, i2)
+
+
+def test_route_policy_mean_against_float64_and_bounds():
+    # the fp32 left-to-right mean stays within a few ulp of the exact mean and between min and max
+    s = synth.normal_scores(500, 12, -0.5, 0.6, 9)
+    _, v, _ = O.route_policy_ref(s.reshape(-1), None, 500, 12, 1, -0.7, agg=O.AGG_MEAN)
+    exact = s.astype(np.float64).mean(axis=1)
+    assert np.abs(v - exact).max() <= 12 * 2.0 ** -23 * np.abs(s).max()
+    assert np.all(v >= s.min(axis=1) - 1e-6) and np.all(v <= s.max(axis=1) + 1e-6)
+    # a block of equal frames has exactly that value as its mean, and min == mean
+    c = np.full((3, 8), -0.625, dtype=np.float32)
+    _, vm, _ = O.route_policy_ref(c.reshape(-1), None, 3, 8, 1, -0.7, agg=O.AGG_MEAN)
+    assert np.all(vm == np.float32(-0.625))
+    # mean >= min always, so at one tau the mean policy accepts a superset of the min policy (Table 2: higher accept rate)
+    a_min, _, _ = O.route_policy_ref(s.reshape(-1), None, 500, 12, 1, -0.7, agg=O.AGG_MIN)
+    a_mean, _, _ = O.route_policy_ref(s.reshape(-1), None, 500, 12, 1, -0.7, agg=O.AGG_MEAN)
+    assert np.all(a_mean >= a_min)
+
+
+def test_route_policy_random_signal_and_accept_stats():
+    B, V = 9 * 400, 400
+    s = synth.normal_scores(B, 12, -0.5, 0.6, 10)
+    u = synth.uniform_scores(B, 1, 0.0, 1.0, 11).reshape(-1)
+    forced, _, _ = O.route_policy_ref(s.reshape(-1), None, B, 12, 0, -0.7, signal=O.SIGNAL_RANDOM, force_first=True,
+                                      blocks_per_video=9, uniforms=u, accept_prob=0.7)
+    plain, _, _ = O.route_policy_ref(s.reshape(-1), None, B, 12, 0, -0.7, signal=O.SIGNAL_RANDOM, force_first=False,
+                                     blocks_per_video=9, uniforms=u, accept_prob=0.7)
+    assert forced.reshape(V, 9)[:, 0].sum() == 0                      # every video's block 0 regenerated
+    assert np.array_equal(forced.reshape(V, 9)[:, 1:], plain.reshape(V, 9)[:, 1:])
+    assert np.array_equal(plain, (u < np.float32(0.7)).astype(np.uint8))   # the scores play no part
+    acc, routable = O.accept_stats_ref(forced, 0, 9)
+    assert routable == 8 * V and acc == int(forced.sum())
+    assert acc / routable == pytest.approx(0.7, abs=0.03)             # matched accept rate (Table 2: 70.3% / 70.0%)
+    # the statistic leaves block 0 out even when it was accepted
+    acc2, routable2 = O.accept_stats_ref(plain, 0, 9)
+    assert routable2 == routable and acc2 == int(plain.reshape(V, 9)[:, 1:].sum())
+    # degenerate probabilities
+    none, _, _ = O.route_policy_ref(s.reshape(-1), None, B, 12, 0, 0.0, signal=O.SIGNAL_RANDOM, uniforms=u, accept_prob=0.0)
+    every, _, _ = O.route_policy_ref(s.reshape(-1), None, B, 12, 0, 0.0, signal=O.SIGNAL_RANDOM, force_first=False,
+                                     uniforms=u, accept_prob=1.0)
+    assert none.sum() == 0 and every.sum() == B
+    # one stream (blocks_per_video = 0): only global block 0 is a first block
+    a1, r1 = O.accept_stats_ref(np.ones(10, dtype=np.uint8), 0, 0)
+    a2, r2 = O.accept_stats_ref(np.ones(10, dtype=np.uint8), 5, 0)
+    assert (a1, r1) == (9, 9) and (a2, r2) == (10, 10)
+    assert O.accept_rate(np.array([1, 1, 0, 1])) == pytest.approx(2 / 3)   # agrees with the older helper
+
+
 # ------------------------------------------------------------------ schedule
 
 def _tiny_provider(sh_d, sh_t, seed):
