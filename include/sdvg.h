@@ -238,6 +238,42 @@ int sdvg_route(const float* scores, const int32_t* frame_offsets,
                int num_blocks, int frames_per_block, int64_t first_block_index, float tau,
                uint8_t* accept, float* q_min, int32_t* argmin, void* stream);
 
+/*
+ * The routing variants of the ablation (Sec. 4.3, Table 2) in one call.
+ *   agg     SDVG_AGG_MIN: worst frame, Eq. (1), exactly as sdvg_route;
+ *           SDVG_AGG_MEAN: "avg-frame scoring": the frames are added left to right in fp32 (every partial
+ *           sum rounded) and the sum is divided by (float)frames with one IEEE division; argmin is -1
+ *   signal  SDVG_SIGNAL_REWARD: accept iff aggregate >= tau;
+ *           SDVG_SIGNAL_RANDOM: "random routing": accept iff uniforms[b] < accept_prob; the scores only
+ *           feed `aggregate`.  The draws are an input (device fp32 [num_blocks], values in [0, 1))
+ *   force_first  non-zero: the first block of a video is rejected whatever the signal says ("force-reject
+ *           + random" against plain "random routing" in Table 2)
+ *   blocks_per_video  0: one stream, only global block 0 is a first block; n > 0: global block g =
+ *           first_block_index + b is a first block iff g % n == 0 (a batch of n-block videos, e.g. the
+ *           paper's 1003 x 9)
+ * accept, aggregate, argmin as in sdvg_route (aggregate takes the place of q_min).
+ * Errors: INVALID_ARG (unknown agg/signal, uniforms NULL with SDVG_SIGNAL_RANDOM, blocks_per_video < 0,
+ * first_block_index < 0 with blocks_per_video > 0), BAD_SHAPE, MISALIGNED.
+ */
+#define SDVG_AGG_MIN       0
+#define SDVG_AGG_MEAN      1
+#define SDVG_SIGNAL_REWARD 0
+#define SDVG_SIGNAL_RANDOM 1
+int sdvg_route_policy(const float* scores, const int32_t* frame_offsets,
+                      int num_blocks, int frames_per_block, int64_t first_block_index, int blocks_per_video,
+                      float tau, int agg, int signal, int force_first,
+                      const float* uniforms, float accept_prob,
+                      uint8_t* accept, float* aggregate, int32_t* argmin, void* stream);
+
+/*
+ * Accept-rate statistics with the convention of Tables 1 and 2 (the always-regenerated first block of a
+ * video is left out): counts[0] = accepted blocks, counts[1] = routable blocks, both over the blocks that
+ * are not first blocks (same first_block_index / blocks_per_video rule as above).  counts: device, two
+ * 64-bit integers, 8-byte aligned; cleared by the call on `stream` before the kernel adds to them.
+ */
+int sdvg_accept_stats(const uint8_t* accept, int num_blocks, int64_t first_block_index, int blocks_per_video,
+                      unsigned long long* counts, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

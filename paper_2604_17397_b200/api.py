@@ -26,6 +26,10 @@ SDVG_ERR_CUDA = 6
 SDVG_ERR_TIMEOUT = 7
 SDVG_STAGE = 1
 SDVG_FINAL = 2
+SDVG_AGG_MIN = 0
+SDVG_AGG_MEAN = 1
+SDVG_SIGNAL_REWARD = 0
+SDVG_SIGNAL_RANDOM = 1
 
 # name -> (restype, argtypes); the list of everything include/sdvg.h declares
 _VP, _I, _I64, _SZ, _F = C.c_void_p, C.c_int, C.c_int64, C.c_size_t, C.c_float
@@ -51,6 +55,8 @@ SIGNATURES = {
     "sdvg_block_attn_status": (_I, [_VP, _VP]),
     "sdvg_block_attn_fwd_noalloc": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, C.POINTER(_VP), _VP]),
     "sdvg_route": (_I, [_VP, _VP, _I, _I, _I64, _F, _VP, _VP, _VP, _VP]),
+    "sdvg_route_policy": (_I, [_VP, _VP, _I, _I, _I64, _I, _F, _I, _I, _I, _VP, _F, _VP, _VP, _VP, _VP]),
+    "sdvg_accept_stats": (_I, [_VP, _I, _I64, _I, _VP, _VP]),
 }
 
 _lib = None
@@ -270,3 +276,30 @@ def sdvg_route(scores, frame_offsets, num_blocks: int, frames_per_block: int, fi
     st = lib().sdvg_route(_ptr(scores), _ptr(frame_offsets), num_blocks, frames_per_block, first_block_index, tau,
                           _ptr(accept), _ptr(q_min), _ptr(argmin), _stream(stream))
     _check(st, "sdvg_route")
+
+
+def sdvg_route_policy(scores, frame_offsets, num_blocks: int, frames_per_block: int, first_block_index: int,
+                      blocks_per_video: int, tau: float, agg: int, signal: int, force_first: bool, uniforms,
+                      accept_prob: float, accept, aggregate, argmin=None, stream=None) -> None:
+    if scores.dtype != torch.float32 or aggregate.dtype != torch.float32 or accept.dtype != torch.uint8:
+        raise ValueError("scores/aggregate must be float32 and accept uint8")
+    if frame_offsets is not None and frame_offsets.dtype != torch.int32:
+        raise ValueError("frame_offsets must be int32")
+    if argmin is not None and argmin.dtype != torch.int32:
+        raise ValueError("argmin must be int32")
+    if uniforms is not None and uniforms.dtype != torch.float32:
+        raise ValueError("uniforms must be float32")
+    st = lib().sdvg_route_policy(_ptr(scores), _ptr(frame_offsets), num_blocks, frames_per_block, first_block_index,
+                                 blocks_per_video, tau, agg, signal, 1 if force_first else 0, _ptr(uniforms),
+                                 accept_prob, _ptr(accept), _ptr(aggregate), _ptr(argmin), _stream(stream))
+    _check(st, "sdvg_route_policy")
+
+
+def sdvg_accept_stats(accept, num_blocks: int, first_block_index: int, blocks_per_video: int, counts,
+                      stream=None) -> None:
+    """counts: device int64 [2] <- (accepted, routable) over the blocks that are not first blocks."""
+    if accept.dtype != torch.uint8 or counts.dtype != torch.int64 or counts.numel() < 2:
+        raise ValueError("accept must be uint8 and counts int64 [2]")
+    st = lib().sdvg_accept_stats(_ptr(accept), num_blocks, first_block_index, blocks_per_video, _ptr(counts),
+                                 _stream(stream))
+    _check(st, "sdvg_accept_stats")

@@ -1,5 +1,7 @@
 // Router (Sec. 3): q_b = min over the block's frame scores (Eq. 1); accept iff q_b >= tau and the
-// block is not global block 0 (forced regeneration of the first block).
+// block is not global block 0 (forced regeneration of the first block).  The same kernel serves the
+// variants of the ablation (Sec. 4.3, Table 2): mean instead of minimum, uniform draws instead of
+// the reward, forcing switched off, first block of every video of a batch.
 //
 // A CTA owns a tile of consecutive blocks, whose scores form one contiguous range.  The range is
 // brought into shared memory with coalesced 16-byte loads (scalar loads for the unaligned head and
@@ -22,7 +24,41 @@ struct RouteParams {
   uint8_t* accept;
   float* q_min;
   int32_t* argmin;
+  int agg, signal, force_first;   // SDVG_AGG_*, SDVG_SIGNAL_*, reject first blocks
+  int blocks_per_video;           // 0: one stream, only global block 0 is a first block
+  const float* uniforms;          // SDVG_SIGNAL_RANDOM: one draw per block
+  float accept_prob;
 };
+
+// Aggregate of frames [s, e) read through `at`: left-to-right strict-'<' minimum, or the fp32 mean
+// (left-to-right sum, every partial sum rounded, then one IEEE division by the frame count).
+template <typename At>
+__device__ __forceinline__ void aggregate(const RouteParams& p, long long s, long long e, At at, float& m, int& idx) {
+  m = __int_as_float(0x7fc00000);
+  idx = -1;
+  if (e <= s) return;
+  m = at(s);
+  if (p.agg == SDVG_AGG_MEAN) {
+    for (long long i = s + 1; i < e; ++i) m = __fadd_rn(m, at(i));
+    m = __fdiv_rn(m, (float)(e - s));
+    return;
+  }
+  idx = 0;
+  for (long long i = s + 1; i < e && m == m; ++i) {
+    const float x = at(i);
+    if (x != x || x < m) { m = x; idx = (int)(i - s); }
+  }
+}
+
+__device__ __forceinline__ void decide(const RouteParams& p, int b, float m, int idx, bool has_frames) {
+  const long long g = p.first_block_index + b;
+  const bool first = p.blocks_per_video > 0 ? (g % p.blocks_per_video == 0) : (g == 0);
+  bool ok = p.signal == SDVG_SIGNAL_RANDOM ? (p.uniforms[b] < p.accept_prob) : (m >= p.tau);
+  ok = ok && has_frames && !(p.force_first && first);
+  p.accept[b] = ok ? 1 : 0;
+  p.q_min[b] = m;
+  if (p.argmin) p.argmin[b] = idx;
+}
 
 __device__ __forceinline__ long long range_begin(const RouteParams& p, int b) {
   return p.offsets ? (long long)p.offsets[b] : (long long)b * p.frames_per_block;
@@ -57,50 +93,64 @@ __global__ void __launch_bounds__(kThreads) route_kernel(const __grid_constant__
       if (b < b1) {
         const int s = (int)(range_begin(p, b) - lo) + shift;
         const int e = (int)(range_begin(p, b + 1) - lo) + shift;
-        float m = __int_as_float(0x7fc00000);
-        int idx = -1;
-        if (e > s) {
-          m = stage[s];
-          idx = 0;
-          for (int i = s + 1; i < e && m == m; ++i) {
-            const float x = stage[i];
-            if (x != x || x < m) { m = x; idx = i - s; }
-          }
-        }
-        const bool ok = (p.first_block_index + b != 0) && (m >= p.tau);
-        p.accept[b] = ok ? 1 : 0;
-        p.q_min[b] = m;
-        if (p.argmin) p.argmin[b] = idx;
+        float m;
+        int idx;
+        aggregate(p, s, e, [&](long long i) { return stage[i]; }, m, idx);
+        decide(p, b, m, idx, e > s);
       }
       __syncthreads();
     } else {
       const int b = b0 + threadIdx.x;
       if (b < b1) {
         const long long s = range_begin(p, b), e = range_begin(p, b + 1);
-        float m = __int_as_float(0x7fc00000);
-        int idx = -1;
-        if (e > s) {
-          m = p.scores[s];
-          idx = 0;
-          for (long long i = s + 1; i < e && m == m; ++i) {
-            const float x = p.scores[i];
-            if (x != x || x < m) { m = x; idx = (int)(i - s); }
-          }
-        }
-        const bool ok = (p.first_block_index + b != 0) && (m >= p.tau);
-        p.accept[b] = ok ? 1 : 0;
-        p.q_min[b] = m;
-        if (p.argmin) p.argmin[b] = idx;
+        float m;
+        int idx;
+        aggregate(p, s, e, [&](long long i) { return p.scores[i]; }, m, idx);
+        decide(p, b, m, idx, e > s);
       }
     }
   }
 }
 
+// accept-rate statistics: counts[0] += accepted, counts[1] += routable, first blocks left out of both
+__global__ void __launch_bounds__(kThreads) accept_stats_kernel(const uint8_t* __restrict__ accept, int num_blocks,
+                                                                 long long first_block_index, int blocks_per_video,
+                                                                 unsigned long long* counts) {
+  unsigned int acc = 0, routable = 0;
+  for (int b = blockIdx.x * kThreads + threadIdx.x; b < num_blocks; b += gridDim.x * kThreads) {
+    const long long g = first_block_index + b;
+    const bool first = blocks_per_video > 0 ? (g % blocks_per_video == 0) : (g == 0);
+    if (!first) {
+      ++routable;
+      acc += accept[b] ? 1u : 0u;
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    acc += __shfl_down_sync(0xffffffffu, acc, o);
+    routable += __shfl_down_sync(0xffffffffu, routable, o);
+  }
+  if ((threadIdx.x & 31) == 0 && (acc | routable)) {
+    atomicAdd(&counts[0], (unsigned long long)acc);
+    atomicAdd(&counts[1], (unsigned long long)routable);
+  }
+}
+
 }  // namespace
 
-extern "C" int sdvg_route(const float* scores, const int32_t* frame_offsets, int num_blocks,
-                          int frames_per_block, int64_t first_block_index, float tau, uint8_t* accept,
-                          float* q_min, int32_t* argmin, void* stream) {
+namespace {
+
+int route_launch(const RouteParams& p, cudaStream_t stream) {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int ntiles = (p.num_blocks + kThreads - 1) / kThreads;
+  const int grid = ntiles < sms * 4 ? ntiles : sms * 4;
+  route_kernel<<<grid, kThreads, 0, stream>>>(p);
+  return sdvg::cuda_status(cudaGetLastError());
+}
+
+int route_checks(const float* scores, const int32_t* frame_offsets, int num_blocks, int frames_per_block,
+                 const uint8_t* accept, const float* q_min, const int32_t* argmin) {
   if (num_blocks < 0) return SDVG_ERR_BAD_SHAPE;
   if (!frame_offsets && frames_per_block < 1) return SDVG_ERR_BAD_SHAPE;
   if (num_blocks == 0) return SDVG_OK;
@@ -109,15 +159,55 @@ extern "C" int sdvg_route(const float* scores, const int32_t* frame_offsets, int
   if ((reinterpret_cast<uintptr_t>(scores) & 3) || (reinterpret_cast<uintptr_t>(q_min) & 3) ||
       (reinterpret_cast<uintptr_t>(frame_offsets) & 3) || (reinterpret_cast<uintptr_t>(argmin) & 3))
     return SDVG_ERR_MISALIGNED;
+  return SDVG_OK;
+}
+
+}  // namespace
+
+extern "C" int sdvg_route(const float* scores, const int32_t* frame_offsets, int num_blocks,
+                          int frames_per_block, int64_t first_block_index, float tau, uint8_t* accept,
+                          float* q_min, int32_t* argmin, void* stream) {
+  int st = route_checks(scores, frame_offsets, num_blocks, frames_per_block, accept, q_min, argmin);
+  if (st != SDVG_OK || num_blocks == 0) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  RouteParams p{scores, frame_offsets, num_blocks, frames_per_block, (long long)first_block_index, tau,
+                accept, q_min, argmin, SDVG_AGG_MIN, SDVG_SIGNAL_REWARD, 1, 0, nullptr, 0.f};
+  return route_launch(p, (cudaStream_t)stream);
+}
+
+extern "C" int sdvg_route_policy(const float* scores, const int32_t* frame_offsets, int num_blocks,
+                                 int frames_per_block, int64_t first_block_index, int blocks_per_video, float tau,
+                                 int agg, int signal, int force_first, const float* uniforms, float accept_prob,
+                                 uint8_t* accept, float* aggregate_out, int32_t* argmin, void* stream) {
+  if ((agg != SDVG_AGG_MIN && agg != SDVG_AGG_MEAN) || (signal != SDVG_SIGNAL_REWARD && signal != SDVG_SIGNAL_RANDOM))
+    return SDVG_ERR_INVALID_ARG;
+  if (blocks_per_video < 0 || (blocks_per_video > 0 && first_block_index < 0)) return SDVG_ERR_INVALID_ARG;
+  int st = route_checks(scores, frame_offsets, num_blocks, frames_per_block, accept, aggregate_out, argmin);
+  if (st != SDVG_OK || num_blocks == 0) return st;
+  if (signal == SDVG_SIGNAL_RANDOM) {
+    if (!uniforms) return SDVG_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(uniforms) & 3) return SDVG_ERR_MISALIGNED;
+  }
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  RouteParams p{scores, frame_offsets, num_blocks, frames_per_block, (long long)first_block_index, tau,
+                accept, aggregate_out, argmin, agg, signal, force_first ? 1 : 0, blocks_per_video, uniforms, accept_prob};
+  return route_launch(p, (cudaStream_t)stream);
+}
+
+extern "C" int sdvg_accept_stats(const uint8_t* accept, int num_blocks, int64_t first_block_index,
+                                 int blocks_per_video, unsigned long long* counts, void* stream_) {
+  if (num_blocks < 0) return SDVG_ERR_BAD_SHAPE;
+  if (!counts || (num_blocks > 0 && !accept)) return SDVG_ERR_INVALID_ARG;
+  if (blocks_per_video < 0 || (blocks_per_video > 0 && first_block_index < 0)) return SDVG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(counts) & 7) return SDVG_ERR_MISALIGNED;
   int st = sdvg::require_sm100();
   if (st != SDVG_OK) return st;
-  RouteParams p{scores, frame_offsets, num_blocks, frames_per_block, (long long)first_block_index, tau,
-                accept, q_min, argmin};
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int ntiles = (num_blocks + kThreads - 1) / kThreads;
-  const int grid = ntiles < sms * 4 ? ntiles : sms * 4;
-  route_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(p);
+  cudaStream_t stream = (cudaStream_t)stream_;
+  cudaError_t e = cudaMemsetAsync(counts, 0, 2 * sizeof(unsigned long long), stream);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  if (num_blocks == 0) return SDVG_OK;
+  const int want = (num_blocks + kThreads - 1) / kThreads;
+  accept_stats_kernel<<<want < 592 ? want : 592, kThreads, 0, stream>>>(accept, num_blocks, (long long)first_block_index,
+                                                                        blocks_per_video, counts);
   return sdvg::cuda_status(cudaGetLastError());
 }
