@@ -339,6 +339,42 @@ def run_ours(args):
     t_route = time_call(lambda: api.sdvg_route(st.scores, None, ROUTE_BLOCKS, ROUTE_FRAMES, 0, -0.7, st.accept,
                                                st.qmin, None))
 
+    # configuration 4 in short: attention at every fill level of the ring (0 .. slots-1 earlier blocks), one cache
+    # filled block by block; each level timed alone over a few launches (burst, not the sustained regime)
+    fill_levels = []
+    if args.workload != "tiny":
+        c2 = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device)
+        for n in range(sh.slots):
+            api.sdvg_kv_commit(c2, st.k_r, st.v, n, api.SDVG_STAGE)
+            t_n = time_call(lambda: api.sdvg_block_attn_fwd(st.q_r, None, None, c2, n, st.out, None, sh.scale, st.ws), n=5)
+            lk_n = (n + 1) * sh.block_tokens
+            fill_levels.append({"prior_blocks": n, "keys": lk_n, "ms": t_n,
+                                "tflops": attn_flops(sh, lk_n) / t_n / 1e9})
+            api.sdvg_kv_commit(c2, st.k_r, st.v, n, api.SDVG_FINAL)
+        c2.close()
+        del c2
+
+    # two problems of this shape in one call (conditional + unconditional pass of guidance): the work items of
+    # both problems share one launch, which is what fills the GPU at the drafter's shape
+    pair = None
+    if args.workload != "tiny":
+        c2 = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device)
+        for n in range(sh.slots - 1):
+            api.sdvg_kv_commit(c2, st.k_r, st.v, n, api.SDVG_FINAL)
+        api.sdvg_kv_commit(c2, st.k_r, st.v, sh.slots - 1, api.SDVG_STAGE)
+        c3 = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device)
+        for n in range(sh.slots - 1):
+            api.sdvg_kv_commit(c3, st.k, st.v, n, api.SDVG_FINAL)
+        api.sdvg_kv_commit(c3, st.k, st.v, sh.slots - 1, api.SDVG_STAGE)
+        out2 = torch.empty_like(st.out)
+        t_pair = time_call(lambda: api.sdvg_block_attn_fwd_batched([st.q_r, st.q], None, None, [c2, c3],
+                                                                   [sh.slots - 1] * 2, [st.out, out2], None,
+                                                                   sh.scale, st.ws), n=10)
+        pair = {"problems": 2, "ms": t_pair, "tflops": 2 * attn_flops(sh, st.lk) / t_pair / 1e9}
+        c2.close()
+        c3.close()
+        del c2, c3, out2
+
     # end to end through the same calls with host buffers: H2D of q,k,v,scores and D2H of out, accept per step,
     # copies of neighbouring steps overlapped with the kernels on separate streams
     st.e2e_setup()
@@ -396,6 +432,8 @@ def run_ours(args):
             "kv_commit": {"ms": t_commit, "gbs": hb["commit"] / t_commit / 1e6,
                           "frac": hb["commit"] / t_commit / 1e6 / pk["hbm_gbs"]},
             "route": {"us": t_route * 1e3, "gbs": hb["route"] / t_route / 1e6}},
+        "attention_by_fill_level": fill_levels,
+        "attention_guidance_pair": pair,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))

@@ -182,6 +182,23 @@ int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self,
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same attention for `batch` independent problems of one shape in one call (at most 4): the two
+ * passes of classifier-free guidance (Sec. 4.1 samples with guidance scale 3.0, i.e. a conditional and an
+ * unconditional pass per denoising step), or several videos.  q, k_self, v_self, caches, block_index, out
+ * and lse are HOST arrays of `batch` entries holding what sdvg_block_attn_fwd takes for one problem
+ * (k_self and v_self may be NULL as arrays = every problem staged; lse may be NULL as an array, or hold
+ * NULL entries).  All caches must have the same block_tokens, heads and head_dim.  Problems whose visible
+ * key segments agree (same ring fill, same staging: the normal case) are processed by ONE launch whose
+ * work items span all problems, which is what fills the GPU at the drafter's shape; otherwise the
+ * problems are launched one after the other on `stream`.  Results are those of `batch` separate calls.
+ * Errors: those of sdvg_block_attn_fwd; BAD_SHAPE for batch > 4 or mismatched cache shapes.
+ */
+int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* const* k_self,
+                                const void* const* v_self, const sdvg_cache* const* caches,
+                                const int64_t* block_index, void* const* out, float* const* lse, float scale,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Synchronises `stream` and reports what the last attention launch that used
  * `workspace` left in its status word: SDVG_OK, or SDVG_ERR_TIMEOUT if a
  * bounded wait inside the kernel gave up (the output is then undefined).

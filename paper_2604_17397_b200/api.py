@@ -52,6 +52,7 @@ SIGNATURES = {
                                    C.POINTER(_I64), _VP]),
     "sdvg_block_attn_workspace_bytes": (_SZ, []),
     "sdvg_block_attn_fwd": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
+    "sdvg_block_attn_fwd_batched": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_attn_status": (_I, [_VP, _VP]),
     "sdvg_block_attn_fwd_noalloc": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, C.POINTER(_VP), _VP]),
     "sdvg_route": (_I, [_VP, _VP, _I, _I, _I64, _F, _VP, _VP, _VP, _VP]),
@@ -238,6 +239,31 @@ def sdvg_block_attn_fwd(q, k_self, v_self, cache: Cache, block_index: int, out, 
                                    _bf16(out, shape), _ptr(lse), scale, workspace.data_ptr(), workspace.numel(),
                                    _stream(stream))
     _check(st, "sdvg_block_attn_fwd")
+
+
+def sdvg_block_attn_fwd_batched(qs, k_selfs, v_selfs, caches, block_indices, outs, lses, scale: float,
+                                workspace: torch.Tensor, stream=None) -> None:
+    """Lists of per-problem arguments (k_selfs / v_selfs / lses may be None = not given for any problem)."""
+    n = len(qs)
+    shape = (caches[0].block_tokens, caches[0].heads, caches[0].head_dim)
+
+    def ptr_array(ts, check):
+        if ts is None:
+            return None
+        return (_VP * n)(*[check(t) for t in ts])
+
+    def lse_ptr(t):
+        if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != (shape[1], shape[0])):
+            raise ValueError("lse must be float32 [heads, block_tokens]")
+        return _ptr(t)
+
+    bf = lambda t: _bf16(t, shape)
+    keep = [ptr_array(qs, bf), ptr_array(k_selfs, bf), ptr_array(v_selfs, bf),
+            (_VP * n)(*[c.handle.value for c in caches]), (_I64 * n)(*block_indices), ptr_array(outs, bf),
+            ptr_array(lses, lse_ptr)]
+    st = lib().sdvg_block_attn_fwd_batched(n, *[C.cast(a, _VP) if a is not None else None for a in keep], scale,
+                                           workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "sdvg_block_attn_fwd_batched")
 
 
 def sdvg_block_attn_status(workspace, stream=None) -> int:

@@ -34,16 +34,26 @@ constexpr int kMaxSegments = 3;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
 constexpr int kWorkspaceBytes = 256;
 
-struct alignas(64) AttnParams {
+constexpr int kMaxBatch = 4;           // independent problems of one shape per launch
+
+// One attention problem of a launch: its tensor maps and outputs.
+struct alignas(64) AttnProblem {
   CUtensorMap q_map;
   CUtensorMap k_map[kMaxSegments];
   CUtensorMap v_map[kMaxSegments];
+  __nv_bfloat16* out;
+  float* lse;
+};
+
+// All problems of a launch have the same shape and the same key segments (same ring fill, same
+// staging); heads of the problems are numbered through: global head g = problem * heads + head.
+struct alignas(64) AttnParams {
+  AttnProblem prob[kMaxBatch];
+  int batch;
   int seg_len[kMaxSegments];
   int nseg;
   int tokens, heads;
   float scale_log2e;                   // scale * log2(e): softmax is evaluated with exp2
-  __nv_bfloat16* out;
-  float* lse;
   unsigned int* work;                  // [0] work counter, [1] status word
 #ifdef SDVG_ATTN_DEBUG
   float* dbg;                          // S, P, O of the first key tile of CTA (0, 0)
@@ -131,6 +141,7 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 3);
   const int tid = threadIdx.x, warp = tid >> 5;
   const int qt = blockIdx.x, head = blockIdx.y;
+  const AttnProblem& pr = p.prob[blockIdx.z];
   constexpr uint32_t kTmemCols = 256;                    // S: [0,128) (P aliases its first 64), O: [128, 128+D)
 
   if (tid == 0) {
@@ -138,7 +149,7 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
     mbar_init(s_bar, 1);
     mbar_init(o_bar, 1);
     fence_mbar_init();
-    prefetch_tmap(&p.q_map);
+    prefetch_tmap(&pr.q_map);
   }
   if (warp == 0) {
     tmem_alloc(tmem_slot, kTmemCols);
@@ -158,7 +169,7 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
   if (tid == 0) {
     mbar_expect_tx(full_bar, L::kTileBytes);
     for (int h = 0; h < L::kHalves; ++h)
-      tma_load_3d(smem + L::kQ + h * L::kPanelBytes, &p.q_map, full_bar, h * 64, qt * kTileM, head);
+      tma_load_3d(smem + L::kQ + h * L::kPanelBytes, &pr.q_map, full_bar, h * 64, qt * kTileM, head);
   }
   alive = wait_bar(full_bar, full_phase, wc);
   full_phase ^= 1;
@@ -177,8 +188,8 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
       if (tid == 0) {
         mbar_expect_tx(full_bar, 2 * L::kTileBytes);
         for (int h = 0; h < L::kHalves; ++h) {
-          tma_load_3d(smem + L::kK + h * L::kPanelBytes, &p.k_map[seg], full_bar, h * 64, kt * kTileN, head);
-          tma_load_3d(smem + L::kV + h * L::kPanelBytes, &p.v_map[seg], full_bar, h * 64, kt * kTileN, head);
+          tma_load_3d(smem + L::kK + h * L::kPanelBytes, &pr.k_map[seg], full_bar, h * 64, kt * kTileN, head);
+          tma_load_3d(smem + L::kV + h * L::kPanelBytes, &pr.v_map[seg], full_bar, h * 64, kt * kTileN, head);
         }
       }
       if (!(alive = wait_bar(full_bar, full_phase, wc))) break;
@@ -291,7 +302,7 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
       tmem_ld32(tO + lane_off + c * 32, o);
       tmem_wait_ld();
       if (row < p.tokens) {
-        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)row * p.heads + head) * D + c * 32);
+        uint4* dst = reinterpret_cast<uint4*>(pr.out + ((size_t)row * p.heads + head) * D + c * 32);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           uint32_t w[4];
@@ -305,8 +316,8 @@ __global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_co
         }
       }
     }
-    if (p.lse && row < p.tokens)
-      p.lse[(size_t)head * p.tokens + row] = m_run * 0.6931471805599453f + logf(l_run);
+    if (pr.lse && row < p.tokens)
+      pr.lse[(size_t)head * p.tokens + row] = m_run * 0.6931471805599453f + logf(l_run);
   }
   tc_fence_before();
   __syncthreads();
@@ -358,7 +369,7 @@ int launch_simple(const AttnParams& p, cudaStream_t stream) {
     if (e != cudaSuccess) return sdvg::cuda_status(e);
     configured = true;
   }
-  dim3 grid((p.tokens + kTileM - 1) / kTileM, p.heads);
+  dim3 grid((p.tokens + kTileM - 1) / kTileM, p.heads, p.batch);
   attn_fwd_simple_kernel<D><<<grid, 128, SimpleSmem<D>::kDynamic, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
 }
@@ -376,7 +387,7 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     configured = true;
   }
-  const WsSchedule sched(p.tokens, p.heads);
+  const WsSchedule sched(p.tokens, p.heads * p.batch);
   const int grid = sched.num_virtual < sms ? sched.num_virtual : sms;
   attn_fwd_ws_kernel<D><<<grid, WsCfg<D>::kThreads, WsCfg<D>::kDynamic, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
@@ -392,32 +403,29 @@ bool use_simple_kernel() {
 }
 
 // Validation, tensor maps, scratch clear and launch shared by the attention entry points.
-int attn_forward(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c, int64_t block_index,
-                 void* out, float* lse, float scale, void* workspace, size_t workspace_bytes,
-                 cudaStream_t stream) {
-  if (!q || !c || !out || !workspace) return SDVG_ERR_INVALID_ARG;
+// Argument and ring-state checks of one problem; touches no CUDA API.
+int check_problem(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c, int64_t block_index,
+                  const void* out, const float* lse) {
+  if (!q || !c || !out) return SDVG_ERR_INVALID_ARG;
   if ((k_self == nullptr) != (v_self == nullptr)) return SDVG_ERR_INVALID_ARG;
-  if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
-  if (!(scale > 0.f) || !isfinite(scale)) return SDVG_ERR_INVALID_ARG;
   if (!sdvg::aligned16(q) || !sdvg::aligned16(k_self) || !sdvg::aligned16(v_self) || !sdvg::aligned16(out) ||
-      (reinterpret_cast<uintptr_t>(lse) & 3) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+      (reinterpret_cast<uintptr_t>(lse) & 3))
     return SDVG_ERR_MISALIGNED;
   if (block_index < 0 || block_index != c->next_block) return SDVG_ERR_BAD_STATE;
   if (!k_self && c->staged_block != block_index) return SDVG_ERR_BAD_STATE;
-  int st = sdvg::require_sm100();
-  if (st != SDVG_OK) return st;
+  return SDVG_OK;
+}
 
+// Fills the tensor maps of one checked problem; the key segments go to seg_len / nseg.
+int fill_problem(AttnProblem& pr, int* seg_len, int* nseg_out, const void* q, const void* k_self, const void* v_self,
+                 const sdvg_cache* c, int64_t block_index, void* out, float* lse) {
   const int T = c->block_tokens, H = c->heads, D = c->head_dim, S = c->slots;
   const size_t row_bytes = (size_t)D * 2;
   const size_t ring_head_stride = (size_t)S * T * row_bytes;
-  AttnParams p = {};
-  p.tokens = T;
-  p.heads = H;
-  p.scale_log2e = scale * 1.4426950408889634f;
-  p.out = (__nv_bfloat16*)out;
-  p.lse = lse;
-  p.work = (unsigned int*)workspace;
-  if ((st = make_map(&p.q_map, q, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+  int st, nseg = 0;
+  pr.out = (__nv_bfloat16*)out;
+  pr.lse = lse;
+  if ((st = make_map(&pr.q_map, q, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
 
   // Visible committed blocks: the last S-1 before block_index, living in slots (b % S).  Their slots
   // form at most two runs of consecutive slots; with the block staged, its slot joins them.
@@ -435,20 +443,62 @@ int attn_forward(const void* q, const void* k_self, const void* v_self, const sd
     if (!use[s]) { ++s; continue; }
     int e = s;
     while (e < S && use[e]) ++e;
-    if (p.nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
+    if (nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
     const long long rows = (long long)(e - s) * T;
     const char* kb = (const char*)c->k_buf + (size_t)s * T * row_bytes;
     const char* vb = (const char*)c->v_buf + (size_t)s * T * row_bytes;
-    if ((st = make_map(&p.k_map[p.nseg], kb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
-    if ((st = make_map(&p.v_map[p.nseg], vb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
-    p.seg_len[p.nseg++] = (int)rows;
+    if ((st = make_map(&pr.k_map[nseg], kb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
+    if ((st = make_map(&pr.v_map[nseg], vb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
+    seg_len[nseg++] = (int)rows;
     s = e;
   }
   if (k_self) {
-    if (p.nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
-    if ((st = make_map(&p.k_map[p.nseg], k_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
-    if ((st = make_map(&p.v_map[p.nseg], v_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
-    p.seg_len[p.nseg++] = T;
+    if (nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
+    if ((st = make_map(&pr.k_map[nseg], k_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+    if ((st = make_map(&pr.v_map[nseg], v_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+    seg_len[nseg++] = T;
+  }
+  *nseg_out = nseg;
+  return SDVG_OK;
+}
+
+// Validation, tensor maps, scratch clear and launch shared by the attention entry points: `batch`
+// problems of one shape, fused into one launch when their key segments agree, else launched one by one.
+int attn_forward_batch(int batch, const void* const* q, const void* const* k_self, const void* const* v_self,
+                       const sdvg_cache* const* caches, const int64_t* block_index, void* const* out,
+                       float* const* lse, float scale, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+  if (batch < 1 || !q || !caches || !block_index || !out || !workspace) return SDVG_ERR_INVALID_ARG;
+  if (batch > kMaxBatch) return SDVG_ERR_BAD_SHAPE;
+  if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
+  if (!(scale > 0.f) || !isfinite(scale)) return SDVG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return SDVG_ERR_MISALIGNED;
+  for (int b = 0; b < batch; ++b) {
+    if (!caches[b]) return SDVG_ERR_INVALID_ARG;
+    if (caches[b]->block_tokens != caches[0]->block_tokens || caches[b]->heads != caches[0]->heads ||
+        caches[b]->head_dim != caches[0]->head_dim)
+      return SDVG_ERR_BAD_SHAPE;
+  }
+  int st;
+  for (int b = 0; b < batch; ++b)
+    if ((st = check_problem(q[b], k_self ? k_self[b] : nullptr, v_self ? v_self[b] : nullptr, caches[b], block_index[b],
+                            out[b], lse ? lse[b] : nullptr)) != SDVG_OK)
+      return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+
+  AttnParams p = {};
+  p.tokens = caches[0]->block_tokens;
+  p.heads = caches[0]->heads;
+  p.scale_log2e = scale * 1.4426950408889634f;
+  p.work = (unsigned int*)workspace;
+  const int D = caches[0]->head_dim;
+  bool same = true;
+  int seg_len[kMaxBatch][kMaxSegments] = {}, nseg[kMaxBatch] = {};
+  for (int b = 0; b < batch; ++b) {
+    st = fill_problem(p.prob[b], seg_len[b], &nseg[b], q[b], k_self ? k_self[b] : nullptr, v_self ? v_self[b] : nullptr,
+                      caches[b], block_index[b], out[b], lse ? lse[b] : nullptr);
+    if (st != SDVG_OK) return st;
+    same = same && nseg[b] == nseg[0];
+    for (int s = 0; same && s < nseg[b]; ++s) same = seg_len[b][s] == seg_len[0][s];
   }
 #ifdef SDVG_ATTN_DEBUG
   p.dbg = workspace_bytes >= (size_t)kWorkspaceBytes + 4 * (128 * 128 + 128 * 64 + 128 * 128)
@@ -457,8 +507,34 @@ int attn_forward(const void* q, const void* k_self, const void* v_self, const sd
 #endif
   cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
   if (e != cudaSuccess) return sdvg::cuda_status(e);
-  if (use_simple_kernel()) return D == 128 ? launch_simple<128>(p, stream) : launch_simple<64>(p, stream);
-  return D == 128 ? launch_ws<128>(p, stream) : launch_ws<64>(p, stream);
+  auto launch = [&](const AttnParams& pp) {
+    if (use_simple_kernel()) return D == 128 ? launch_simple<128>(pp, stream) : launch_simple<64>(pp, stream);
+    return D == 128 ? launch_ws<128>(pp, stream) : launch_ws<64>(pp, stream);
+  };
+  if (same) {
+    p.batch = batch;
+    p.nseg = nseg[0];
+    for (int s = 0; s < nseg[0]; ++s) p.seg_len[s] = seg_len[0][s];
+    return launch(p);
+  }
+  // different ring fill or staging per problem: one launch each, in stream order (they share the status word)
+  for (int b = 0; b < batch; ++b) {
+    AttnParams one = p;
+    one.prob[0] = p.prob[b];
+    one.batch = 1;
+    one.nseg = nseg[b];
+    for (int s = 0; s < kMaxSegments; ++s) one.seg_len[s] = seg_len[b][s];
+    if ((st = launch(one)) != SDVG_OK) return st;
+  }
+  return SDVG_OK;
+}
+
+int attn_forward(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c, int64_t block_index,
+                 void* out, float* lse, float scale, void* workspace, size_t workspace_bytes,
+                 cudaStream_t stream) {
+  if (!c) return SDVG_ERR_INVALID_ARG;
+  return attn_forward_batch(1, &q, k_self ? &k_self : nullptr, v_self ? &v_self : nullptr, &c, &block_index, &out,
+                            &lse, scale, workspace, workspace_bytes, stream);
 }
 
 // Scratch for sdvg_block_attn_fwd_noalloc: lives in the library image, one copy per device that
@@ -481,6 +557,14 @@ int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, c
                         size_t workspace_bytes, void* stream_) {
   return attn_forward(q, k_self, v_self, c, block_index, out, lse, scale, workspace, workspace_bytes,
                       (cudaStream_t)stream_);
+}
+
+int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* const* k_self,
+                                const void* const* v_self, const sdvg_cache* const* caches,
+                                const int64_t* block_index, void* const* out, float* const* lse, float scale,
+                                void* workspace, size_t workspace_bytes, void* stream_) {
+  return attn_forward_batch(batch, q, k_self, v_self, caches, block_index, out, lse, scale, workspace,
+                            workspace_bytes, (cudaStream_t)stream_);
 }
 
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,

@@ -261,10 +261,12 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       mbar_init(&kv_empty[s], 1);
     }
     fence_mbar_init();
-    prefetch_tmap(&p.q_map);
-    for (int s = 0; s < p.nseg; ++s) {
-      prefetch_tmap(&p.k_map[s]);
-      prefetch_tmap(&p.v_map[s]);
+    for (int b = 0; b < p.batch; ++b) {
+      prefetch_tmap(&p.prob[b].q_map);
+      for (int s = 0; s < p.nseg; ++s) {
+        prefetch_tmap(&p.prob[b].k_map[s]);
+        prefetch_tmap(&p.prob[b].v_map[s]);
+      }
     }
   }
   if (warp == 0) {
@@ -278,7 +280,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
   // Every wait of this kernel gives up at the same absolute time; a thread that gives up records
   // the timeout and leaves its role loop, and all roles meet at the common exit below.
   const Deadline dl{globaltimer_ns() + kWaitLimitNs, p.work + 1};
-  const WsSchedule sched(p.tokens, p.heads);
+  const WsSchedule sched(p.tokens, p.heads * p.batch);     // it.head[] are global heads: problem * heads + head
   int ntiles_k = 0;
   for (int s = 0; s < p.nseg; ++s) ntiles_k += (p.seg_len[s] + kTileN - 1) / kTileN;
 
@@ -305,10 +307,11 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         SDVG_TRACE(4, kv_issued);
         if (leader) {
           mbar_expect_tx(&kv_full[ring.stage], C::kTileBytes);
-          const CUtensorMap* m = is_v ? &p.v_map[seg] : &p.k_map[seg];
+          const AttnProblem& pr = p.prob[head / p.heads];
+          const CUtensorMap* m = is_v ? &pr.v_map[seg] : &pr.k_map[seg];
           for (int h = 0; h < C::kHalves; ++h)
             tma_load_3d(smem + C::kKV + ring.stage * C::kTileBytes + h * C::kPanelBytes, m, &kv_full[ring.stage],
-                        h * 64, kt * kTileN, head);
+                        h * 64, kt * kTileN, head % p.heads);
         }
         ring.template advance<C::kStages>();
         ++kv_issued;
@@ -326,8 +329,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           if (leader) {
             mbar_expect_tx(&q_full[i], C::kTileBytes);
             for (int h = 0; h < C::kHalves; ++h)
-              tma_load_3d(smem + C::kQ + i * C::kTileBytes + h * C::kPanelBytes, &p.q_map, &q_full[i], h * 64,
-                          it.tile[i] * kTileM, it.head[i]);
+              tma_load_3d(smem + C::kQ + i * C::kTileBytes + h * C::kPanelBytes, &p.prob[it.head[i] / p.heads].q_map,
+                          &q_full[i], h * 64, it.tile[i] * kTileM, it.head[i] % p.heads);
           }
         }
         // K/V tiles in the order the issuer consumes them
@@ -688,7 +691,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       if (!(alive = wait_bar(&o_full[i], (pv_cnt - 1) & 1, dl))) break;
       tc_fence_after();
       const int grow = it.tile[i] * kTileM + row;
-      const int head = it.head[i];
+      const AttnProblem& pr = p.prob[it.head[i] / p.heads];
+      const int head = it.head[i] % p.heads;
       const float inv = 1.f / l_run;
 #pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {                  // once per item: keep its code small
@@ -696,7 +700,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         tmem_ld32(tO + c * 32, o);
         tmem_wait_ld();
         if (grow < p.tokens) {
-          uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)grow * p.heads + head) * D + c * 32);
+          uint4* dst = reinterpret_cast<uint4*>(pr.out + ((size_t)grow * p.heads + head) * D + c * 32);
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             uint32_t w[4];
@@ -711,8 +715,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         }
       }
       tc_fence_before();
-      if (p.lse && grow < p.tokens)
-        p.lse[(size_t)head * p.tokens + grow] = -neg * 0.6931471805599453f + logf(l_run);
+      if (pr.lse && grow < p.tokens)
+        pr.lse[(size_t)head * p.tokens + grow] = -neg * 0.6931471805599453f + logf(l_run);
     }
   }
 

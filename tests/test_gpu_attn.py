@@ -171,3 +171,53 @@ def test_config3_wan14b_shape_fused_prologue_cache_bits_and_sampled_attention():
         o_ref, lse_ref = O.block_attn_ref(qr_ref, kr_ref, v, ref, b, sh.scale, heads=[h], rows=rows)
         check(got[rows, h], o_ref[:, 0], ("wan14b", h))
         assert np.allclose(lse_h[h, rows], lse_ref[0], rtol=0, atol=2e-3)
+
+
+def test_batched_call_equals_separate_calls_and_the_oracle():
+    # cond / uncond pair of one shape: one launch over both problems; bit-identical to two separate calls
+    sh = synth.Shape("pair", heads=3, head_dim=128, frames=1, grid_h=12, grid_w=25, slots=3)
+    caches = [api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim) for _ in range(2)]
+    refs = [O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim) for _ in range(2)]
+    ws = api.attn_workspace()
+    for b in range(4):
+        qkv = [[synth.block_tensor(sh, 60 + n, b, 0, t) for t in (synth.Q, synth.K, synth.V)] for n in range(2)]
+        dev = [[to_dev(x) for x in prob] for prob in qkv]
+        for n in range(2):
+            api.sdvg_kv_commit(caches[n], dev[n][1], dev[n][2], b, api.SDVG_STAGE)
+        outs = [torch.full_like(dev[n][0], float("nan")) for n in range(2)]
+        lses = [torch.full((sh.heads, sh.block_tokens), float("nan"), device="cuda") for _ in range(2)]
+        api.sdvg_block_attn_fwd_batched([d[0] for d in dev], None, None, caches, [b, b], outs, lses, sh.scale, ws)
+        assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+        for n in range(2):
+            one = torch.empty_like(outs[n])
+            api.sdvg_block_attn_fwd(dev[n][0], None, None, caches[n], b, one, None, sh.scale, ws)
+            assert torch.equal(one.view(torch.int16), outs[n].view(torch.int16))
+            o_ref, lse_ref = O.block_attn_ref(*qkv[n], refs[n], b, sh.scale)
+            check(to_bits(outs[n]), o_ref, ("batched", b, n))
+            assert np.allclose(lses[n].cpu().numpy(), lse_ref, rtol=0, atol=2e-3)
+            api.sdvg_kv_commit(caches[n], dev[n][1], dev[n][2], b, api.SDVG_FINAL)
+            refs[n].commit(b, qkv[n][1], qkv[n][2], O.FINAL)
+
+
+def test_batched_call_with_different_ring_fill_falls_back_to_separate_launches():
+    sh = synth.Shape("pair2", heads=2, head_dim=64, frames=1, grid_h=10, grid_w=20, slots=3)
+    caches = [api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim) for _ in range(2)]
+    refs = [O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim) for _ in range(2)]
+    ws = api.attn_workspace()
+    k0, v0 = synth.block_tensor(sh, 70, 0, 0, synth.K), synth.block_tensor(sh, 70, 0, 0, synth.V)
+    api.sdvg_kv_commit(caches[1], to_dev(k0), to_dev(v0), 0, api.SDVG_FINAL)     # problem 1 is one block ahead
+    refs[1].commit(0, k0, v0, O.FINAL)
+    blocks = [0, 1]
+    qkv = [[synth.block_tensor(sh, 71 + n, blocks[n], 0, t) for t in (synth.Q, synth.K, synth.V)] for n in range(2)]
+    dev = [[to_dev(x) for x in prob] for prob in qkv]
+    outs = [torch.empty_like(dev[n][0]) for n in range(2)]
+    api.sdvg_block_attn_fwd_batched([d[0] for d in dev], [d[1] for d in dev], [d[2] for d in dev], caches, blocks,
+                                    outs, None, sh.scale, ws)
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    for n in range(2):
+        o_ref, _ = O.block_attn_ref(*qkv[n], refs[n], blocks[n], sh.scale)
+        check(to_bits(outs[n]), o_ref, ("fallback", n))
+    with pytest.raises(api.SdvgError) as e:
+        api.sdvg_block_attn_fwd_batched([dev[0][0]] * 5, None, None, [caches[0]] * 5, [0] * 5, [outs[0]] * 5, None,
+                                        sh.scale, ws)
+    assert e.value.status == api.SDVG_ERR_BAD_SHAPE
