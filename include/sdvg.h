@@ -206,6 +206,16 @@ int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* con
 int sdvg_block_attn_status(const void* workspace, void* stream);
 
 /*
+ * Self-test of the bounded device-side wait (no counterpart in the paper; it backs the promise that a
+ * stuck attention kernel returns instead of hanging the GPU).  Launches one warp that waits, through the
+ * wait the attention kernel uses, for an mbarrier phase that nothing will ever complete, with a limit of
+ * limit_ns nanoseconds (1 .. 1e9).  The warp must give up after the limit, record SDVG_ERR_TIMEOUT in the
+ * status word of `workspace` and exit normally; sdvg_block_attn_status(workspace) then returns
+ * SDVG_ERR_TIMEOUT and the context stays usable.  workspace: as for sdvg_block_attn_fwd.
+ */
+int sdvg_selftest_bounded_wait(void* workspace, size_t workspace_bytes, unsigned long long limit_ns, void* stream);
+
+/*
  * Same computation as sdvg_block_attn_fwd for callers that cannot allocate device memory
  * (the paper has no counterpart; this is a deployment convenience).  Some hosts of this
  * library run under a fixed memory plan: an inference server that hands every byte of HBM
@@ -290,6 +300,17 @@ int sdvg_route_policy(const float* scores, const int32_t* frame_offsets,
  */
 int sdvg_accept_stats(const uint8_t* accept, int num_blocks, int64_t first_block_index, int blocks_per_video,
                       unsigned long long* counts, void* stream);
+
+/* ---- speculative state: snapshot and restore ------------------------------ */
+/*
+ * Copies `count` device buffers (at most 64) in one launch: dst[i][0 .. bytes[i]) = src[i][0 .. bytes[i]).
+ * Sec. 3 "Inference flow": the decoder's cache is cloned before a draft block is decoded and scored, and
+ * restored when the router rejects the block; the snapshot is this call, the restore the same call with
+ * src and dst exchanged.  src, dst and bytes are HOST arrays; the buffers are device memory, 16-byte aligned,
+ * every length a multiple of 16; a source must not overlap a destination.
+ * Errors: BAD_SHAPE (count outside 0..64, a length not a multiple of 16), INVALID_ARG, MISALIGNED.
+ */
+int sdvg_state_copy(const void* const* src, void* const* dst, const size_t* bytes, int count, void* stream);
 
 #ifdef __cplusplus
 }

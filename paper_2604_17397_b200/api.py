@@ -53,11 +53,13 @@ SIGNATURES = {
     "sdvg_block_attn_workspace_bytes": (_SZ, []),
     "sdvg_block_attn_fwd": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_attn_fwd_batched": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
+    "sdvg_selftest_bounded_wait": (_I, [_VP, _SZ, C.c_ulonglong, _VP]),
     "sdvg_block_attn_status": (_I, [_VP, _VP]),
     "sdvg_block_attn_fwd_noalloc": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, C.POINTER(_VP), _VP]),
     "sdvg_route": (_I, [_VP, _VP, _I, _I, _I64, _F, _VP, _VP, _VP, _VP]),
     "sdvg_route_policy": (_I, [_VP, _VP, _I, _I, _I64, _I, _F, _I, _I, _I, _VP, _F, _VP, _VP, _VP, _VP]),
     "sdvg_accept_stats": (_I, [_VP, _I, _I64, _I, _VP, _VP]),
+    "sdvg_state_copy": (_I, [_VP, _VP, _VP, _I, _VP]),
 }
 
 _lib = None
@@ -266,6 +268,11 @@ def sdvg_block_attn_fwd_batched(qs, k_selfs, v_selfs, caches, block_indices, out
     _check(st, "sdvg_block_attn_fwd_batched")
 
 
+def sdvg_selftest_bounded_wait(workspace: torch.Tensor, limit_ns: int, stream=None) -> None:
+    st = lib().sdvg_selftest_bounded_wait(workspace.data_ptr(), workspace.numel(), limit_ns, _stream(stream))
+    _check(st, "sdvg_selftest_bounded_wait")
+
+
 def sdvg_block_attn_status(workspace, stream=None) -> int:
     """`workspace` is the tensor given to sdvg_block_attn_fwd, or the integer device address
     returned by sdvg_block_attn_fwd_noalloc."""
@@ -329,3 +336,19 @@ def sdvg_accept_stats(accept, num_blocks: int, first_block_index: int, blocks_pe
     st = lib().sdvg_accept_stats(_ptr(accept), num_blocks, first_block_index, blocks_per_video, _ptr(counts),
                                  _stream(stream))
     _check(st, "sdvg_accept_stats")
+
+
+def sdvg_state_copy(srcs, dsts, stream=None) -> None:
+    """dsts[i] <- srcs[i] for lists of contiguous CUDA tensors of equal byte sizes (snapshot or restore)."""
+    n = len(srcs)
+    if len(dsts) != n:
+        raise ValueError("srcs and dsts must have the same length")
+    nbytes = []
+    for a, b in zip(srcs, dsts):
+        if a.numel() * a.element_size() != b.numel() * b.element_size():
+            raise ValueError("source and destination sizes differ")
+        nbytes.append(a.numel() * a.element_size())
+    st = lib().sdvg_state_copy(C.cast((_VP * n)(*[_ptr(t) for t in srcs]), _VP),
+                               C.cast((_VP * n)(*[_ptr(t) for t in dsts]), _VP),
+                               C.cast((_SZ * n)(*nbytes), _VP), n, _stream(stream))
+    _check(st, "sdvg_state_copy")

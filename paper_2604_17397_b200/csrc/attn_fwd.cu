@@ -537,6 +537,20 @@ int attn_forward(const void* q, const void* k_self, const void* v_self, const sd
                             &lse, scale, workspace, workspace_bytes, stream);
 }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier phase that nothing ever completes, with
+// the given time limit, through the same wait_bar the attention kernel uses.
+__global__ void bounded_wait_selftest_kernel(unsigned int* work, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const Deadline dl{globaltimer_ns() + limit_ns, work + 1};
+  const bool ok = wait_warp(&bar, 0, dl);
+  if (threadIdx.x == 0) work[0] = ok ? 1u : 2u;          // 2: the wait gave up, as it should
+}
+
 // Scratch for sdvg_block_attn_fwd_noalloc: lives in the library image, one copy per device that
 // loads it.  In host code this name is only a handle for cudaGetSymbolAddress, never a pointer.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kWorkspaceBytes];
@@ -594,6 +608,19 @@ int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v
   if (scratch_device_ptr) *scratch_device_ptr = scratch;
   return attn_forward(q, k_self, v_self, c, block_index, out, lse, scale, scratch, sizeof(g_noalloc_scratch),
                       (cudaStream_t)stream_);
+}
+
+int sdvg_selftest_bounded_wait(void* workspace, size_t workspace_bytes, unsigned long long limit_ns, void* stream_) {
+  if (!workspace || workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return SDVG_ERR_MISALIGNED;
+  if (limit_ns == 0 || limit_ns > 1000000000ull) return SDVG_ERR_INVALID_ARG;     // at most one second
+  int st = sdvg::require_sm100();
+  if (st != SDVG_OK) return st;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>((unsigned int*)workspace, limit_ns);
+  return sdvg::cuda_status(cudaGetLastError());
 }
 
 int sdvg_block_attn_status(const void* workspace, void* stream_) {

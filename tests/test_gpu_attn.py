@@ -221,3 +221,22 @@ def test_batched_call_with_different_ring_fill_falls_back_to_separate_launches()
         api.sdvg_block_attn_fwd_batched([dev[0][0]] * 5, None, None, [caches[0]] * 5, [0] * 5, [outs[0]] * 5, None,
                                         sh.scale, ws)
     assert e.value.status == api.SDVG_ERR_BAD_SHAPE
+
+
+def test_bounded_wait_gives_up_reports_timeout_and_leaves_the_context_usable():
+    import time
+    ws = api.attn_workspace()
+    t0 = time.perf_counter()
+    api.sdvg_selftest_bounded_wait(ws, 20_000_000)                   # 20 ms limit on a phase nothing completes
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_ERR_TIMEOUT    # synchronises the stream
+    dt = time.perf_counter() - t0
+    assert 0.015 <= dt < 1.0, dt
+    assert int(ws.view(torch.int32)[0].item()) == 2                  # the waiting warp ran to its end
+    # the device still works: a normal attention call on the same workspace succeeds and clears the status
+    sh = synth.TINY
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    q, k, v = (to_dev(synth.block_tensor(sh, 80, 0, 0, t)) for t in (synth.Q, synth.K, synth.V))
+    out = torch.empty_like(q)
+    api.sdvg_block_attn_fwd(q, k, v, cache, 0, out, None, sh.scale, ws)
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    assert torch.isfinite(out.float()).all()
