@@ -14,8 +14,8 @@
 // Tensor-pipe order per key tile j:  PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1); while the pipe works for
 // lane 1 the softmax warps of lane 0 turn S_0(j+1) into P_0(j+1), and vice versa.  The running row
 // maximum is only raised when it grew by more than 2^8 in the exp2 domain, so O is rarely rescaled
-// and the correction warps stay off the critical path; the final 1/l normalisation and the store
-// are done by the softmax warps themselves, which own the same TMEM lanes.
+// and that work stays off the critical path; the final 1/l normalisation and the store are done by
+// the softmax warps themselves, which own the same TMEM lanes.
 //
 // The chain S ready -> softmax -> P ready -> PV, QK -> next S ready of one lane sets the pace, so it
 // is shortened from both ends.  A softmax thread reduces its whole row of S to the maximum, hands
@@ -25,13 +25,18 @@
 // the PV product on the first part while the softmax thread finishes the third quarter.  The issuer
 // is blocked while the tensor pipe's queue is full, so it looks at the K/V stages of its next step
 // right after queueing a batch of MMAs, when that costs nothing.  The producer and issuer warps
-// run their loops with all 32 lanes (warp-uniform control flow and values) and only predicate the TMA / MMA / commit instructions on one elected lane:
-// descriptors and addresses then stay in uniform registers.
+// run their loops with all 32 lanes (warp-uniform control flow and values) and only predicate the
+// TMA / MMA / commit instructions on one elected lane: descriptors and addresses then stay in
+// uniform registers.  All role loops are kept small (rare paths rolled, ragged tiles masked in
+// tensor memory by a cold loop): the roles share the SM's instruction cache, and the issuer, which
+// runs once per key tile, pays for every line the others push out.
 //
 // The exponentials are the co-limiter of this kernel: a 128 x 128 tile needs 16384 of them and the
 // special-function unit delivers 16 per clock per SM, the same 1024 clocks the tile's two MMAs take.
-// A compile-time share of the elements can therefore be evaluated on the FMA pipe instead (range
-// reduction to [0, 1) plus a cubic, relative error 2e-4, a tenth of the bf16 rounding P gets anyway).
+// A compile-time share of the elements can be evaluated on the FMA pipe instead (range reduction to
+// [0, 1) plus a cubic, relative error 2e-4, a tenth of the bf16 rounding P gets anyway); it is off by
+// default (SDVG_ATTN_POLY_PAIRS = 0) because the extra instructions cost more than the freed
+// special-function slots gain once the GPU runs under its power cap.
 #pragma once
 
 #ifdef SDVG_ATTN_TRACE
@@ -523,56 +528,54 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
       #pragma unroll 1
       for (int j = 0; j < ntiles_k && alive; ++j) {
-        {
 #pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            if (i >= it.lanes || !alive) break;
-            const uint32_t par = cnt[i] & 1;
-            if (!(alive = wait_bar(&row_ready[i], par, dl))) break;
-            const float neg = s_neg[i * 128 + row];
-            // the row's reference maximum moved iff -m*c2 changed; both sides derive the factor the same way
-            const bool moved = (j > 0) && (neg != neg_prev[i]);
-            const float alpha = moved ? fast_exp2(__fsub_rn(neg, neg_prev[i])) : 1.f;
-            neg_prev[i] = neg;
-            SDVG_TRACE(3, 1000 * i + j);
-            if (__any_sync(0xffffffffu, moved)) {
-              // PV_i(j-1) is commit number cnt[i] - 1 on o_full[i]
-              if (!(alive = wait_bar(&o_full[i], (cnt[i] - 1) & 1, dl))) break;
-              tc_fence_after();
-#pragma unroll 1
-              for (int c = 0; c < D / 32; ++c) {          // rare path: keep its code small
-                uint32_t o[32];
-                tmem_ld32(tO[i] + c * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-                tmem_st32(tO[i] + c * 32, o);
-              }
-              tmem_wait_st();
-              tc_fence_before();
-              l_part[i] *= alpha;
-            }
-            SDVG_TRACE(3, 20000 + 1000 * i + j);
-            // ---- this row's share of P: key columns 96-127 -------------------------------------
+        for (int i = 0; i < 2; ++i) {
+          if (i >= it.lanes || !alive) break;
+          const uint32_t par = cnt[i] & 1;
+          if (!(alive = wait_bar(&row_ready[i], par, dl))) break;
+          const float neg = s_neg[i * 128 + row];
+          // the row's reference maximum moved iff -m*c2 changed; both sides derive the factor the same way
+          const bool moved = (j > 0) && (neg != neg_prev[i]);
+          const float alpha = moved ? fast_exp2(__fsub_rn(neg, neg_prev[i])) : 1.f;
+          neg_prev[i] = neg;
+          SDVG_TRACE(3, 1000 * i + j);
+          if (__any_sync(0xffffffffu, moved)) {
+            // PV_i(j-1) is commit number cnt[i] - 1 on o_full[i]
+            if (!(alive = wait_bar(&o_full[i], (cnt[i] - 1) & 1, dl))) break;
             tc_fence_after();
-            uint32_t s3[32], pk[16];
-            tmem_ld32(tS[i] + 96, s3);
-            tmem_wait_ld();
-            uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-            exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
-            tmem_st16(tS[i] + 48, pk);
-            {
-              float a0, a1, b0, b1;
-              unpack2(sum_a, a0, a1);
-              unpack2(sum_b, b0, b1);
-              l_part[i] += (a0 + a1) + (b0 + b1);
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {          // rare path: keep its code small
+              uint32_t o[32];
+              tmem_ld32(tO[i] + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+              tmem_st32(tO[i] + c * 32, o);
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&p_lo[i]);
-            SDVG_TRACE(3, 30000 + 1000 * i + j);
-            ++cnt[i];
+            l_part[i] *= alpha;
           }
+          SDVG_TRACE(3, 20000 + 1000 * i + j);
+          // ---- this row's share of P: key columns 96-127 -------------------------------------
+          tc_fence_after();
+          uint32_t s3[32], pk[16];
+          tmem_ld32(tS[i] + 96, s3);
+          tmem_wait_ld();
+          uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
+          exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
+          tmem_st16(tS[i] + 48, pk);
+          {
+            float a0, a1, b0, b1;
+            unpack2(sum_a, a0, a1);
+            unpack2(sum_b, b0, b1);
+            l_part[i] += (a0 + a1) + (b0 + b1);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&p_lo[i]);
+          SDVG_TRACE(3, 30000 + 1000 * i + j);
+          ++cnt[i];
         }
       }
       if (!alive) break;
