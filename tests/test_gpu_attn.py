@@ -240,3 +240,33 @@ def test_bounded_wait_gives_up_reports_timeout_and_leaves_the_context_usable():
     api.sdvg_block_attn_fwd(q, k, v, cache, 0, out, None, sh.scale, ws)
     assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
     assert torch.isfinite(out.float()).all()
+
+
+def test_rising_logits_rescale_the_accumulator_at_almost_every_key_tile():
+    # Keys whose magnitude grows along the sequence: the row maximum keeps rising by more than the lazy-rescale
+    # threshold, so the helper warps rescale O (and both partial row sums) again and again.
+    sh = synth.Shape("rising", heads=2, head_dim=128, frames=3, grid_h=16, grid_w=16, slots=3)   # 768 tokens = 6 key tiles per block
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    ws = api.attn_workspace()
+    for b in range(3):
+        q = synth.block_tensor(sh, 90, b, 0, synth.Q, std=1.0)
+        # all queries share a direction with the keys so that logits grow with the key index
+        base = O.bf16_to_f64(synth.block_tensor(sh, 90, 0, 1, synth.K))[0:1, :, :]
+        ramp = (1.0 + 10.0 * (np.arange(sh.block_tokens) + b * sh.block_tokens) / (3 * sh.block_tokens))[:, None, None]
+        k = O.f64_to_bf16(base * ramp + 0.05 * O.bf16_to_f64(synth.block_tensor(sh, 90, b, 0, synth.K)))
+        q = O.f64_to_bf16(np.abs(O.bf16_to_f64(q)) * np.sign(base) * 1.5)
+        v = synth.block_tensor(sh, 90, b, 0, synth.V)
+        dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
+        out = torch.full_like(dq, float("nan"))
+        lse = torch.full((sh.heads, sh.block_tokens), float("nan"), device="cuda")
+        api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_STAGE)
+        api.sdvg_block_attn_fwd(dq, None, None, cache, b, out, lse, sh.scale, ws)
+        assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+        o_ref, lse_ref = O.block_attn_ref(q, k, v, ref, b, sh.scale)
+        # the logits of one row span far more than 2^8 between the first and the last key tile
+        assert (lse_ref.max() - lse_ref.min()) >= 0 and np.isfinite(lse_ref).all()
+        check(to_bits(out), o_ref, ("rising", b))
+        assert np.allclose(lse.cpu().numpy(), lse_ref, rtol=2e-4, atol=2e-3)
+        api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_FINAL)
+        ref.commit(b, k, v, O.FINAL)
