@@ -3,8 +3,8 @@
  *
  * The library implements what every drafter and target denoising step of SDVG
  * (speculative decoding for block-autoregressive video diffusion) pays in its
- * attention backbone (Sec. 4.1 "Models": causal attention with KV caching via
- * RoPE, bf16) plus the routing rule of Sec. 3:
+ * attention backbone (Sec. 4.1 "Models": causal attention over a KV cache, rotary
+ * positions, bf16) plus the routing rule of Sec. 3:
  *
  *   sdvg_rope3d_qk        3D rotary embedding (frame, row, column) of q and k
  *   sdvg_block_attn_fwd   a block of latent frames attends to itself (all keys

@@ -60,7 +60,7 @@ def f64_to_bf16(x: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
-# 3D RoPE  (Sec. 4.1 "KV caching via RoPE positional embeddings")
+# 3D RoPE  (Sec. 4.1 "Models": the backbone carries positions by rotary embeddings)
 # --------------------------------------------------------------------------
 
 
@@ -410,7 +410,7 @@ def route_policy_ref(scores, frame_offsets, num_blocks: int, frames_per_block: i
 
 def accept_stats_ref(accept, first_block_index: int = 0, blocks_per_video: int = 0):
     """(accepted, routable) block counts, the first block of every video left out of both
-    (accept-rate convention of Tables 1 and 2: "excludes block 0 (always force-rejected)")."""
+    (accept-rate convention stated in the captions of Tables 1 and 2: the always-regenerated block 0 is not counted)."""
     a = np.asarray(accept).astype(np.int64)
     g = np.arange(a.size, dtype=np.int64) + first_block_index
     first = (g == 0) if blocks_per_video == 0 else (g % blocks_per_video == 0)

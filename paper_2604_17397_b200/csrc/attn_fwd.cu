@@ -1,5 +1,5 @@
 // Block attention forward for sm_100a: O = softmax(scale * Q K^T) V over every visible key
-// (Sec. 4.1: causal attention backbone with KV caching; no key is masked inside a call because the
+// (Sec. 4.1 "Models": both models attend causally over a KV cache; no key is masked inside a call because the
 // block sees all of itself and all of its window).
 //
 // Both products run on the 5th-generation tensor cores (tcgen05.mma, bf16 in, fp32 accumulators in
