@@ -163,9 +163,9 @@ size_t sdvg_block_attn_workspace_bytes(void);
  * out[i, h, :] = sum_j softmax_j(scale * <q[i,h,:], K[j,h,:]>) V[j,h,:] where j
  * runs over every token of the committed blocks visible to block_index (the
  * last slots-1 blocks before it) and of block_index itself; no key is masked:
- * bidirectional inside the block, causal across blocks (Sec. 4.1 "causal
- * attention backbone with KV caching"; Sec. 1: blocks condition on earlier
- * content through the shared cache).
+ * bidirectional inside the block, causal across blocks (Sec. 4.1 "Models": both
+ * models attend causally over a KV cache; Sec. 1: a block is conditioned on
+ * earlier content through that cache).
  *   q, out        device bf16 [block_tokens, heads, head_dim] of the cache's shape
  *   k_self/v_self device bf16, same shape, the block's own roped K and V; both
  *                 NULL means the block was staged (SDVG_STAGE) and is read from the ring
