@@ -30,7 +30,7 @@ METRIC = "block-attn TFLOP/s per denoise step @14B shape (% bf16 peak); KV-commi
 ROUTE_BLOCKS = 1003 * 9          # the paper's evaluation volume: 1003 videos x 9 blocks (Sec. 4.1)
 ROUTE_FRAMES = 12
 # DRAM bytes (read + write) of ONE attention launch, from an ncu capture of the kernel as it stands
-# (profiles/attn_fwd_ws_14b_dram.md); None for workloads that were not captured.
+# (its summary is kept with the other profiler summaries); None for workloads that were not captured.
 ATTN_DRAM_BYTES_PER_LAUNCH = {"14b": 1.394e9}
 CPU_SAMPLE_HEADS = 12           # heads of one step the CPU oracle is timed on (about 10-20 s of host work)
 
