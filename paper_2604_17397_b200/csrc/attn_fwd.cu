@@ -387,8 +387,8 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     configured = true;
   }
-  const WsSchedule sched(p.tokens, p.heads * p.batch);
-  const int grid = sched.num_virtual < sms ? sched.num_virtual : sms;
+  const int total_tiles = ((p.tokens + kTileM - 1) / kTileM) * p.heads * p.batch;
+  const int grid = total_tiles < sms ? total_tiles : sms;
   attn_fwd_ws_kernel<D><<<grid, WsCfg<D>::kThreads, WsCfg<D>::kDynamic, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
 }

@@ -1,7 +1,7 @@
 // Warp-specialised, persistent block-attention kernel (included by attn_fwd.cu after the common
 // definitions).  One CTA per SM; a work item is a pair of 128-row query tiles ("lanes").  Usually
-// the two tiles belong to one head and share every K/V tile; when the tile count of a head is odd,
-// the last tiles of two heads form an item whose lanes stream their own K/V.
+// the two tiles belong to one head and share every K/V tile; a pair that straddles a head boundary
+// has lanes that stream their own K/V, and the tiles left over after the pairs run alone.
 //
 //   warps 0-3   softmax of lane 0 (one thread per row)            \  S, P and O live in tensor memory:
 //   warps 4-7   softmax of lane 1                                  >  S0 S1 O0 O1 = 4 x 128 columns
@@ -85,32 +85,33 @@ struct WsItem {
   bool dual;              // lanes stream their own K/V (different heads)
 };
 
-// Static schedule: virtual item v < num_pairs is pair v of consecutive tiles of one head; each later
-// item takes the last (unpaired) tiles of two heads.  Every item costs the same, so a round-robin
-// over the CTAs is balanced.
+// Static schedule.  The query tiles of all heads form one list (head-major); with G CTAs and U tiles,
+// the first P = G * floor(U / 2G) items are pairs of neighbouring tiles (tiles 2v and 2v+1: the same
+// head, or, where the pair straddles a head boundary, two heads whose lanes stream their own K/V),
+// the remaining U - 2P tiles are items of one tile each.  Items are dealt round-robin, so every CTA
+// gets the same number of pairs, CTAs that run at the same time work on neighbouring tiles of few
+// heads (their K/V tiles are shared through L2), and the single tiles even out the last round.
 struct WsSchedule {
-  int tiles, pairs_per_head, num_pairs, num_singles, num_virtual;
-  __host__ __device__ WsSchedule(int tokens, int heads) {
+  int tiles, num_pairs, num_items;
+  __host__ __device__ WsSchedule(int tokens, int heads, int ctas) {
     tiles = (tokens + kTileM - 1) / kTileM;
-    pairs_per_head = tiles / 2;
-    num_pairs = pairs_per_head * heads;
-    num_singles = (tiles & 1) ? heads : 0;
-    num_virtual = num_pairs + (num_singles + 1) / 2;
+    const int total = tiles * heads;
+    num_pairs = (total / (2 * ctas)) * ctas;
+    num_items = num_pairs + (total - 2 * num_pairs);
   }
   __device__ void get(int v, WsItem& it) const {
+    const int g0 = v < num_pairs ? 2 * v : 2 * num_pairs + (v - num_pairs);
+    it.head[0] = g0 / tiles;
+    it.tile[0] = g0 - it.head[0] * tiles;
     if (v < num_pairs) {
-      const int h = v / pairs_per_head;
-      it.head[0] = it.head[1] = h;
-      it.tile[0] = 2 * (v - h * pairs_per_head);
-      it.tile[1] = it.tile[0] + 1;
+      it.head[1] = (g0 + 1) / tiles;
+      it.tile[1] = g0 + 1 - it.head[1] * tiles;
       it.lanes = 2;
-      it.dual = false;
+      it.dual = it.head[1] != it.head[0];
     } else {
-      const int s = 2 * (v - num_pairs);
-      it.head[0] = s;
-      it.head[1] = s + 1;
-      it.tile[0] = it.tile[1] = tiles - 1;
-      it.lanes = (s + 1 < num_singles) ? 2 : 1;
+      it.head[1] = it.head[0];
+      it.tile[1] = it.tile[0];
+      it.lanes = 1;
       it.dual = true;
     }
   }
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
   // Every wait of this kernel gives up at the same absolute time; a thread that gives up records
   // the timeout and leaves its role loop, and all roles meet at the common exit below.
   const Deadline dl{globaltimer_ns() + kWaitLimitNs, p.work + 1};
-  const WsSchedule sched(p.tokens, p.heads * p.batch);     // it.head[] are global heads: problem * heads + head
+  const WsSchedule sched(p.tokens, p.heads * p.batch, gridDim.x);   // it.head[] are global heads: problem * heads + head
   int ntiles_k = 0;
   for (int s = 0; s < p.nseg; ++s) ntiles_k += (p.seg_len[s] + kTileN - 1) / kTileN;
 
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       };
 
       #pragma unroll 1
-      for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
+      for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
         WsItem it;
         sched.get(v, it);
 #pragma unroll
@@ -411,7 +412,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       };
 
       #pragma unroll 1
-      for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
+      for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
         WsItem it;
         sched.get(v, it);
         const int nl = it.lanes;
@@ -522,7 +523,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && tid == 256)
     #pragma unroll 1
-    for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
+    for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
       WsItem it;
       sched.get(v, it);
       float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
@@ -601,7 +602,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0)
     #pragma unroll 1
-    for (int v = blockIdx.x; v < sched.num_virtual && alive; v += gridDim.x) {
+    for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
       WsItem it;
       sched.get(v, it);
       if (it.lanes <= i) continue;
