@@ -69,7 +69,8 @@ struct WsCfg {
   static constexpr int kQ = 0;                                      // two query tiles
   static constexpr int kKV = 2 * kTileBytes;
   static constexpr int kRowState = kKV + kStages * kTileBytes;      // float [2][128]: -m*c2 of a row, later the helper's l
-  static constexpr int kBars = kRowState + 2 * 128 * 4;
+  static constexpr int kMerge = kRowState + 2 * 128 * 4;            // float [128]: lane 1's -m*c2 when a split tile is merged
+  static constexpr int kBars = kMerge + 128 * 4;
   static constexpr int kNumBars = 20 + 2 * kStages;
   static constexpr int kMisc = kBars + kNumBars * 8;                // tmem slot
   static constexpr int kTotal = kMisc + 16;
@@ -82,15 +83,21 @@ struct WsCfg {
 struct WsItem {
   int head[2], tile[2];   // per lane
   int lanes;              // 1 or 2
-  bool dual;              // lanes stream their own K/V (different heads)
+  bool dual;              // lanes stream their own K/V tiles (different heads, or one tile split by keys)
+  bool split;             // both lanes work on ONE query tile: lane i takes key tiles i, i + 2, i + 4, ...
+  int nk[2];              // key tiles per lane
+  // branch-free on purpose: a loop-invariant branch on `split` makes the compiler clone whole role loops
+  __device__ int key_tile(int lane, int t) const { return (t << (int)split) + (lane & -(int)split); }
 };
 
 // Static schedule.  The query tiles of all heads form one list (head-major); with G CTAs and U tiles,
 // the first P = G * floor(U / 2G) items are pairs of neighbouring tiles (tiles 2v and 2v+1: the same
 // head, or, where the pair straddles a head boundary, two heads whose lanes stream their own K/V),
-// the remaining U - 2P tiles are items of one tile each.  Items are dealt round-robin, so every CTA
-// gets the same number of pairs, CTAs that run at the same time work on neighbouring tiles of few
-// heads (their K/V tiles are shared through L2), and the single tiles even out the last round.
+// the remaining U - 2P tiles are items of one tile each, whose keys are split between the two lanes
+// (even and odd key tiles; the two partial results are merged when the item ends), so that a single
+// tile costs about half a pair.  Items are dealt round-robin, so every CTA gets the same number of
+// pairs, CTAs that run at the same time work on neighbouring tiles of few heads (their K/V tiles are
+// shared through L2), and the single tiles even out the last round.
 struct WsSchedule {
   int tiles, num_pairs, num_items;
   __host__ __device__ WsSchedule(int tokens, int heads, int ctas) {
@@ -99,7 +106,7 @@ struct WsSchedule {
     num_pairs = (total / (2 * ctas)) * ctas;
     num_items = num_pairs + (total - 2 * num_pairs);
   }
-  __device__ void get(int v, WsItem& it) const {
+  __device__ void get(int v, int ntiles_k, WsItem& it) const {
     const int g0 = v < num_pairs ? 2 * v : 2 * num_pairs + (v - num_pairs);
     it.head[0] = g0 / tiles;
     it.tile[0] = g0 - it.head[0] * tiles;
@@ -108,11 +115,16 @@ struct WsSchedule {
       it.tile[1] = g0 + 1 - it.head[1] * tiles;
       it.lanes = 2;
       it.dual = it.head[1] != it.head[0];
+      it.split = false;
+      it.nk[0] = it.nk[1] = ntiles_k;
     } else {
       it.head[1] = it.head[0];
       it.tile[1] = it.tile[0];
-      it.lanes = 1;
+      it.split = ntiles_k >= 2;
+      it.lanes = it.split ? 2 : 1;
       it.dual = true;
+      it.nk[0] = it.split ? (ntiles_k + 1) / 2 : ntiles_k;
+      it.nk[1] = it.split ? ntiles_k / 2 : 0;
     }
   }
 };
@@ -236,6 +248,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
   // share of the row sum travels back through the same word
   float* s_neg = reinterpret_cast<float*>(smem + C::kRowState);
   float* s_lhelp = s_neg;
+  float* s_merge = reinterpret_cast<float*>(smem + C::kMerge);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBars);
   uint64_t* q_full = bars;            // [2] TMA -> MMA
   uint64_t* q_empty = bars + 2;       // [2] MMA -> TMA
@@ -245,6 +258,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
   uint64_t* row_ready = bars + 12;    // [2] softmax -> helper: -m*c2 of the row published, 128 arrivals
   uint64_t* o_full = bars + 14;       // [2] MMA -> helper / softmax epilogue
   uint64_t* l_ready = bars + 16;      // [2] helper -> softmax epilogue: its share of the row sum, 128 arrivals
+  uint64_t* lane1_done = bars + 18;   // softmax of lane 1 -> softmax of lane 0: partial result of a split tile published, 128 arrivals
+  uint64_t* merge_done = bars + 19;   // softmax of lane 0 -> softmax of lane 1: O_1 has been read, 128 arrivals
   uint64_t* kv_full = bars + 20;      // [kStages]
   uint64_t* kv_empty = kv_full + C::kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kMisc);
@@ -262,6 +277,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       mbar_init(&o_full[i], 1);
       mbar_init(&l_ready[i], 128);
     }
+    mbar_init(lane1_done, 128);
+    mbar_init(merge_done, 128);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&kv_full[s], 1);
       mbar_init(&kv_empty[s], 1);
@@ -326,7 +343,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       #pragma unroll 1
       for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
         WsItem it;
-        sched.get(v, it);
+        sched.get(v, ntiles_k, it);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           if (i >= it.lanes || !alive) break;
@@ -339,14 +356,16 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
                           &q_full[i], h * 64, it.tile[i] * kTileM, it.head[i] % p.heads);
           }
         }
-        // K/V tiles in the order the issuer consumes them
+        // K/V tiles in the order the issuer consumes them: K of the first key tile of every stream, then
+        // step by step and lane by lane V of this step and K of the next
         const int streams = it.dual ? it.lanes : 1;
-        for (int s = 0; s < streams && alive; ++s) load_kv(false, it.head[s], 0);
+        for (int s = 0; s < streams && alive; ++s) load_kv(false, it.head[s], it.key_tile(s, 0));
         #pragma unroll 1
-        for (int j = 0; j < ntiles_k && alive; ++j)
+        for (int t = 0; t < it.nk[0] && alive; ++t)
           for (int s = 0; s < streams && alive; ++s) {
-            load_kv(true, it.head[s], j);
-            if (j + 1 < ntiles_k && alive) load_kv(false, it.head[s], j + 1);
+            if (t >= it.nk[s]) continue;
+            load_kv(true, it.head[s], it.key_tile(s, t));
+            if (t + 1 < it.nk[s] && alive) load_kv(false, it.head[s], it.key_tile(s, t + 1));
           }
       }
       // Drain: every load issued above lands in this CTA's shared memory; do not exit under them.
@@ -414,9 +433,10 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       #pragma unroll 1
       for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
         WsItem it;
-        sched.get(v, it);
+        sched.get(v, ntiles_k, it);
         const int nl = it.lanes;
         const bool dual = it.dual;
+        const int nk0 = it.nk[0], nk1 = it.nk[1];      // scalars: indexing the item by the lane would put it in local memory
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           if (i >= nl || !alive) break;
@@ -442,19 +462,23 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             if (last_user) mma_commit(&kv_empty[stK]);
           }
         }
-        // ---- main loop -------------------------------------------------------------------------
+        // ---- main loop: step t of lane i works on that lane's t-th key tile --------------------------
         bool filled = false;               // the stages of the coming step were seen filled already
         #pragma unroll 1
-        for (int j = 0; j < ntiles_k && alive; ++j) {
-          const bool more = j + 1 < ntiles_k;
+        for (int t = 0; t < nk0 && alive; ++t) {
           uint32_t stV = 0;
-          SDVG_TRACE(2, 100 + j);
+          SDVG_TRACE(2, 100 + t);
+          // everything that depends on t alone is worked out here: each instruction inside the lane loop
+          // sits between "P is ready" and the next MMA
+          const int nl_t = t < nk1 ? nl : 1;                 // a split tile with an odd number of key tiles ends on lane 0
+          const bool more0 = t + 1 < nk0, more1 = t + 1 < nk1;
 #pragma unroll 1
-          for (int i = 0; i < nl && alive; ++i) {
+          for (int i = 0; i < nl_t && alive; ++i) {
+            const bool more = i == 0 ? more0 : more1;
             const bool own = (i == 0) || dual;
             const bool last_user = dual || (i == nl - 1);
             if (own) {
-              // V_j and K_(j+1)
+              // V of this step and K of the next
               stV = ring.stage;
               const uint32_t phV = ring.phase;
               if (!filled) filled = stages_filled(more ? 2 : 1);
@@ -471,27 +495,27 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
               }
               filled = false;
             }
-            SDVG_TRACE(2, 1000 + i * 1000 + j);
+            SDVG_TRACE(2, 1000 + i * 1000 + t);
             const uint32_t par = (pv_par >> i) & 1;
             pv_par ^= 1u << i;
-            // P_i(j) columns 0-63 and 96-127 stored, O_i rescaled (for j = 0: O_i was read out by the
+            // P_i columns 0-63 and 96-127 stored, O_i rescaled (for t = 0: O_i was read out by the
             // epilogue of the previous item before its softmax threads arrived here)
             if (!(alive = wait_warp(&p_lo[i], par, dl))) break;
-            SDVG_TRACE(2, 3000 + i * 1000 + j);
+            SDVG_TRACE(2, 3000 + i * 1000 + t);
             tc_fence_after();
             if (leader) {
-              issue_pv(i, stV, 6, 8, j > 0 ? 1u : 0u);
+              issue_pv(i, stV, 6, 8, t > 0 ? 1u : 0u);
               issue_pv(i, stV, 0, 4, 1u);
             }
-            // six MMAs are queued: a good moment to look at the stages of the next step that takes any
+            // six MMAs are queued: a good moment to look at the stages of the next step, if it takes any
             {
-              const bool next_in_this_j = dual && (i + 1 < nl);
-              const bool next_more = next_in_this_j ? more : (j + 2 < ntiles_k);
-              if ((next_in_this_j || (last_user && more)) && (dual || i == nl - 1))
+              const bool next_in_this_t = dual && (i + 1 < nl_t);
+              const bool next_more = next_in_this_t ? more1 : (t + 2 < nk0);
+              if ((next_in_this_t || (last_user && more0)) && (dual || i == nl_t - 1))
                 filled = stages_filled(next_more ? 2 : 1);
             }
             if (!(alive = wait_warp(&p_mid[i], par, dl))) break;
-            SDVG_TRACE(2, 5000 + i * 1000 + j);
+            SDVG_TRACE(2, 5000 + i * 1000 + t);
             tc_fence_after();
             if (leader) {
               issue_pv(i, stV, 4, 6, 1u);
@@ -505,7 +529,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
                 mma_commit(&q_empty[i]);
               }
             }
-            SDVG_TRACE(2, 9000 + i * 1000 + j);
+            SDVG_TRACE(2, 9000 + i * 1000 + t);
           }
         }
       }
@@ -525,13 +549,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     #pragma unroll 1
     for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
       WsItem it;
-      sched.get(v, it);
+      sched.get(v, ntiles_k, it);
       float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
       #pragma unroll 1
-      for (int j = 0; j < ntiles_k && alive; ++j) {
+      for (int j = 0; j < it.nk[0] && alive; ++j) {          // step j of lane i: that lane's j-th key tile
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           if (i >= it.lanes || !alive) break;
+          if (j >= it.nk[i]) continue;
           const uint32_t par = cnt[i] & 1;
           if (!(alive = wait_bar(&row_ready[i], par, dl))) break;
           const float neg = s_neg[i * 128 + row];
@@ -598,23 +623,35 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     const uint32_t tO = tmem_base + 256 + i * 128 + lane_off;
     const float c2 = p.scale_log2e;
     const uint64_t c2x2 = pack2(c2, c2);
-    uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0;
+    uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0, split_cnt = 0;
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0)
     #pragma unroll 1
     for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
       WsItem it;
-      sched.get(v, it);
+      sched.get(v, ntiles_k, it);
       if (it.lanes <= i) continue;
+      // this lane's fields as scalars (indexing the item by the lane would put it in local memory)
+      const int my_nk = i == 0 ? it.nk[0] : it.nk[1];
+      const int my_tile = i == 0 ? it.tile[0] : it.tile[1];
+      const int my_head = i == 0 ? it.head[0] : it.head[1];
       float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2
-      int j = 0;
-      #pragma unroll 1
-      for (int seg = 0; seg < p.nseg && alive; ++seg) {
-        const int len = p.seg_len[seg];
-        const int nt = (len + kTileN - 1) / kTileN;
+      {
         #pragma unroll 1
-        for (int kt = 0; kt < nt && alive; ++kt, ++j) {
-          const int valid = min(kTileN, len - kt * kTileN);
+        for (int j = 0; j < my_nk && alive; ++j) {        // this lane's j-th key tile
+          // number of real keys in that tile: the last tile of a key segment may be ragged
+          int valid = kTileN;
+          {
+            int kt = it.key_tile(i, j);
+            for (int seg = 0; seg < p.nseg; ++seg) {
+              const int nt = (p.seg_len[seg] + kTileN - 1) / kTileN;
+              if (kt < nt) {
+                valid = min(kTileN, p.seg_len[seg] - kt * kTileN);
+                break;
+              }
+              kt -= nt;
+            }
+          }
           SDVG_TRACE(i, 0 + j);
           if (!(alive = wait_bar(&s_full[i], s_cnt & 1, dl))) break;
           SDVG_TRACE(i, 1000 + j);
@@ -691,18 +728,55 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       if (!(alive = wait_bar(&l_ready[i], item_cnt & 1, dl))) break;
       ++item_cnt;
       l_run += s_lhelp[i * 128 + row];
-      pv_cnt += ntiles_k;
+      pv_cnt += my_nk;
       if (!(alive = wait_bar(&o_full[i], (pv_cnt - 1) & 1, dl))) break;
       tc_fence_after();
-      const int grow = it.tile[i] * kTileM + row;
-      const AttnProblem& pr = p.prob[it.head[i] / p.heads];
-      const int head = it.head[i] % p.heads;
+      // A split tile: both lanes hold a partial result of the SAME rows over disjoint keys, each relative to its
+      // own reference maximum.  Lane 1 publishes (-m*c2, l) and waits until lane 0 has folded O_1 into its output.
+      float w0 = 1.f, w1 = 0.f;                      // weights of O_0 and O_1 in the merged numerator
+      if (it.split) {
+        const uint32_t par = split_cnt & 1;
+        ++split_cnt;
+        if (i == 1) {
+          s_merge[row] = neg;
+          s_neg[128 + row] = l_run;
+          tc_fence_before();
+          mbar_arrive(lane1_done);
+          alive = wait_bar(merge_done, par, dl);
+          if (!alive) break;
+          continue;
+        }
+        if (!(alive = wait_bar(lane1_done, par, dl))) break;
+        tc_fence_after();
+        const float neg1 = s_merge[row], l1 = s_neg[128 + row];
+        const float negm = fminf(neg, neg1);         // the larger of the two reference maxima
+        w0 = fast_exp2(negm - neg);                  // 2^((m_0 - m) c2) <= 1: rebases lane 0's sums to the common maximum
+        w1 = fast_exp2(negm - neg1);
+        l_run = l_run * w0 + l1 * w1;
+        neg = negm;
+      }
+      const int grow = my_tile * kTileM + row;
+      const AttnProblem& pr = p.prob[my_head / p.heads];
+      const int head = my_head % p.heads;
       const float inv = 1.f / l_run;
+      w0 *= inv;
+      w1 *= inv;
 #pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {                  // once per item: keep its code small
         uint32_t o[32];
         tmem_ld32(tO + c * 32, o);
         tmem_wait_ld();
+        if (it.split) {
+          uint32_t o1[32];
+          tmem_ld32(tO + 128 + c * 32, o1);               // O_1 sits 128 columns after O_0, same TMEM lanes
+          tmem_wait_ld();
+#pragma unroll
+          for (int k = 0; k < 32; ++k)
+            o[k] = __float_as_uint(__uint_as_float(o[k]) * w0 + __uint_as_float(o1[k]) * w1);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * w0);
+        }
         if (grow < p.tokens) {
           uint4* dst = reinterpret_cast<uint4*>(pr.out + ((size_t)grow * p.heads + head) * D + c * 32);
 #pragma unroll
@@ -710,8 +784,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             uint32_t w[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(o[q4 * 8 + 2 * k]) * inv,
-                                                       __uint_as_float(o[q4 * 8 + 2 * k + 1]) * inv);
+              __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(o[q4 * 8 + 2 * k]),
+                                                       __uint_as_float(o[q4 * 8 + 2 * k + 1]));
               w[k] = *reinterpret_cast<uint32_t*>(&b);
             }
             dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -719,6 +793,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         }
       }
       tc_fence_before();
+      if (it.split) mbar_arrive(merge_done);
       if (pr.lse && grow < p.tokens)
         pr.lse[(size_t)head * p.tokens + grow] = -neg * 0.6931471805599453f + logf(l_run);
     }
