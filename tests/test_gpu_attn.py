@@ -270,3 +270,11 @@ def test_rising_logits_rescale_the_accumulator_at_almost_every_key_tile():
         assert np.allclose(lse.cpu().numpy(), lse_ref, rtol=2e-4, atol=2e-3)
         api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_FINAL)
         ref.commit(b, k, v, O.FINAL)
+
+
+@pytest.mark.parametrize("slots", [1, 2])
+@pytest.mark.parametrize("staged", [False, True])
+def test_smallest_rings(slots, staged):
+    # slots = 1: a block sees only itself; slots = 2: itself and the block before it
+    sh = synth.Shape(f"ring{slots}", heads=2, head_dim=64, frames=1, grid_h=9, grid_w=17, slots=slots)
+    run_sequence(sh, 4, 95 + slots, staged)
