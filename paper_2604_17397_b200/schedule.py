@@ -124,3 +124,40 @@ def run_schedule(num_blocks: int, steps: int, scores: torch.Tensor, tau: float,
     res.accept = accept_d.cpu().numpy()
     res.q_min = qmin_d.cpu().numpy()
     return res
+
+
+class BlockStepGraph:
+    """The S denoising steps of ONE block captured into a CUDA graph (Sec. 4.1: 4 steps per block).
+
+    Every step is the fused rope + stage call followed by the attention call, reading q, k, v from
+    fixed input tensors (``self.q[s]``, ``self.k[s]``, ``self.v[s]``: fill them before ``replay``) and
+    writing ``self.out[s]``.  The ring state does not change inside the loop (SDVG_STAGE leaves it
+    alone), so the captured launches stay valid until the block's final commit; a new block needs a
+    new capture because its ring slot, frame offset and key segments differ.  One eager pass runs
+    first: the library's one-time set-up (kernel attributes, device queries) must not happen during
+    capture.
+    """
+
+    def __init__(self, m: ModelState, block: int, steps: int):
+        shape = (m.cache.block_tokens, m.cache.heads, m.cache.head_dim)
+        dev = m.table.device
+        new = lambda: torch.zeros(shape, dtype=torch.bfloat16, device=dev)
+        self.q, self.k, self.v = ([new() for _ in range(steps)] for _ in range(3))
+        self.q_roped = [new() for _ in range(steps)]
+        self.out = [new() for _ in range(steps)]
+        self.m, self.block, self.steps = m, block, steps
+        self._run()                                   # warm-up, eager
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self._run()
+
+    def _run(self):
+        m, b = self.m, self.block
+        for s in range(self.steps):
+            api.sdvg_rope3d_qk_commit(m.cache, self.q[s], self.k[s], self.v[s], self.q_roped[s], None, m.grid,
+                                      b * m.frames, m.table, m.tab_frames, b, api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd(self.q_roped[s], None, None, m.cache, b, self.out[s], None, m.scale, m.workspace)
+
+    def replay(self):
+        self.graph.replay()

@@ -200,3 +200,34 @@ def test_config5_trace_full_shapes_iid_scores():
         assert np.array_equal(acc.cpu().numpy(), a)
         vecs.append(a.tobytes())
     run_trace(synth.WAN_1_3B, synth.WAN_14B, B, iid, -0.7, 53)
+
+
+def test_block_steps_replayed_from_a_cuda_graph_equal_the_eager_calls():
+    sh = synth.Shape("graph", heads=3, head_dim=128, frames=3, grid_h=6, grid_w=11, slots=3)
+    tabf = 4 * sh.frames
+    m = model_state(sh, tabf)
+    grid = (sh.frames, sh.grid_h, sh.grid_w)
+    for b in range(3):                                  # block 2 sees two committed blocks
+        if b == 2:
+            g = schedule.BlockStepGraph(m, b, STEPS)
+            eager = []
+            for s in range(STEPS):
+                q, k, v = (to_dev(synth.block_tensor(sh, 97, b, s, t)) for t in (synth.Q, synth.K, synth.V))
+                g.q[s].copy_(q); g.k[s].copy_(k); g.v[s].copy_(v)
+                api.sdvg_rope3d_qk_commit(m.cache, q, k, v, m.q_roped, None, grid, b * sh.frames, m.table, tabf, b,
+                                          api.SDVG_STAGE)
+                api.sdvg_block_attn_fwd(m.q_roped, None, None, m.cache, b, m.out, None, sh.scale, m.workspace)
+                eager.append(m.out.clone())
+            for o in g.out:
+                o.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            assert api.sdvg_block_attn_status(m.workspace) == api.SDVG_OK
+            for s in range(STEPS):
+                assert torch.equal(g.out[s].view(torch.int16), eager[s].view(torch.int16)), s
+            g.replay()                                  # a second replay gives the same bits again
+            torch.cuda.synchronize()
+            assert torch.equal(g.out[STEPS - 1].view(torch.int16), eager[STEPS - 1].view(torch.int16))
+        k, v = (to_dev(synth.block_tensor(sh, 97, b, 9, t)) for t in (synth.K, synth.V))
+        api.sdvg_rope3d_qk_commit(m.cache, None, k, v, None, None, grid, b * sh.frames, m.table, tabf, b, api.SDVG_FINAL)
+    m.cache.close()
