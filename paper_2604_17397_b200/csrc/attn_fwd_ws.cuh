@@ -386,18 +386,18 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       bool alive = true;
       SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
 
-      // The issue loops are deliberately not unrolled: this warp runs through its code once per key
-      // tile, between long stretches of other warps' code, and every instruction it does not have
-      // is one it does not have to fetch again.
+      // Every instruction this warp executes between "P is ready" and the MMAs lengthens the chain that
+      // paces the kernel, so the issue loops are unrolled (descriptor offsets become immediates) while the
+      // loop over the two lanes stays rolled to keep the code this warp has to fetch small.
       // S_i = Q_i K^T into TMEM columns [128 i, 128 i + 128)
       auto issue_qk = [&](int i, uint32_t st) {
         const uint32_t d = tmem_base + i * 128;
         uint64_t a = smem_desc_sw128(sQ + i * C::kTileBytes, 16, 1024);
         uint64_t b = smem_desc_sw128(sKV + st * C::kTileBytes, 16, 1024);
         uint32_t acc = 0;
-#pragma unroll 1
+#pragma unroll
         for (int h = 0; h < C::kHalves; ++h) {
-#pragma unroll 1
+#pragma unroll
           for (int k4 = 0; k4 < 4; ++k4) {
             mma_ss(d, a + 2 * k4, b + 2 * k4, kIdescQK, acc);          // 16 bf16 = 32 B = 2 descriptor units
             acc = 1;
@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       auto issue_pv = [&](int i, uint32_t st, int k0, int k1, uint32_t acc) {
         const uint32_t d = tmem_base + 256 + i * 128, a = tmem_base + i * 128;
         uint64_t b = smem_desc_sw128(sKV + st * C::kTileBytes, C::kPanelBytes, 1024) + (uint64_t)(k0 * (2048 >> 4));
-#pragma unroll 1
+#pragma unroll
         for (int kk = k0; kk < k1; ++kk) {
           mma_ts(d, a + kk * 8, b, kIdescPV, acc);
           acc = 1;
