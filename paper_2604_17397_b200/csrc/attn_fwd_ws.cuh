@@ -463,7 +463,24 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           }
         }
         // ---- main loop: step t of lane i works on that lane's t-th key tile --------------------------
-        bool filled = false;               // the stages of the coming step were seen filled already
+        // The stages of a step (V of this key tile, K of the next) are taken from the ring one step ahead, in
+        // the shadow of MMAs already queued: what is left at the start of a step is a look at `nx.filled`.
+        struct {
+          uint32_t stV, phV, stK, phK;
+          bool filled;
+        } nx = {0, 0, 0, 0, false};
+        auto take = [&](bool with_k) {
+          nx.stV = ring.stage;
+          nx.phV = ring.phase;
+          nx.filled = stages_filled(with_k ? 2 : 1);
+          ring.template advance<C::kStages>();
+          if (with_k) {
+            nx.stK = ring.stage;
+            nx.phK = ring.phase;
+            ring.template advance<C::kStages>();
+          }
+        };
+        take(nk0 > 1);                                       // for step (0, lane 0)
         #pragma unroll 1
         for (int t = 0; t < nk0 && alive; ++t) {
           uint32_t stV = 0;
@@ -475,25 +492,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
 #pragma unroll 1
           for (int i = 0; i < nl_t && alive; ++i) {
             const bool more = i == 0 ? more0 : more1;
-            const bool own = (i == 0) || dual;
             const bool last_user = dual || (i == nl - 1);
-            if (own) {
-              // V of this step and K of the next
-              stV = ring.stage;
-              const uint32_t phV = ring.phase;
-              if (!filled) filled = stages_filled(more ? 2 : 1);
-              ring.template advance<C::kStages>();
-              uint32_t phK = 0;
-              if (more) {
-                stK = ring.stage;
-                phK = ring.phase;
-                ring.template advance<C::kStages>();
+            if (i == 0 || dual) {                            // this lane has stages of its own
+              stV = nx.stV;
+              stK = nx.stK;
+              if (!nx.filled) {
+                if (!(alive = wait_warp(&kv_full[stV], nx.phV, dl))) break;
+                if (more && !(alive = wait_warp(&kv_full[stK], nx.phK, dl))) break;
               }
-              if (!filled) {
-                if (!(alive = wait_warp(&kv_full[stV], phV, dl))) break;
-                if (more && !(alive = wait_warp(&kv_full[stK], phK, dl))) break;
-              }
-              filled = false;
             }
             SDVG_TRACE(2, 1000 + i * 1000 + t);
             const uint32_t par = (pv_par >> i) & 1;
@@ -507,12 +513,11 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
               issue_pv(i, stV, 6, 8, t > 0 ? 1u : 0u);
               issue_pv(i, stV, 0, 4, 1u);
             }
-            // six MMAs are queued: a good moment to look at the stages of the next step, if it takes any
+            // six MMAs are queued: take the stages of the next step that has stages of its own
             {
               const bool next_in_this_t = dual && (i + 1 < nl_t);
-              const bool next_more = next_in_this_t ? more1 : (t + 2 < nk0);
-              if ((next_in_this_t || (last_user && more0)) && (dual || i == nl_t - 1))
-                filled = stages_filled(next_more ? 2 : 1);
+              if (next_in_this_t) take(more1);
+              else if (more0 && (dual || i == nl_t - 1)) take(t + 2 < nk0);
             }
             if (!(alive = wait_warp(&p_mid[i], par, dl))) break;
             SDVG_TRACE(2, 5000 + i * 1000 + t);
