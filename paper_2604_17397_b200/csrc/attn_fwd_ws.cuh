@@ -390,32 +390,33 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       // paces the kernel, so the issue loops are unrolled (descriptor offsets become immediates) while the
       // loop over the two lanes stays rolled to keep the code this warp has to fetch small.
       // S_i = Q_i K^T into TMEM columns [128 i, 128 i + 128)
+      // Descriptors of stage 0 and of the two query tiles, built once; a stage or a 16-wide slice is then one
+      // addition to the address field (all of this CTA's shared memory fits that field, so nothing carries out).
+      const uint64_t descQ0 = smem_desc_sw128(sQ, 16, 1024);
+      const uint64_t descK0 = smem_desc_sw128(sKV, 16, 1024);
+      const uint64_t descV0 = smem_desc_sw128(sKV, C::kPanelBytes, 1024);
       auto issue_qk = [&](int i, uint32_t st) {
         const uint32_t d = tmem_base + i * 128;
-        uint64_t a = smem_desc_sw128(sQ + i * C::kTileBytes, 16, 1024);
-        uint64_t b = smem_desc_sw128(sKV + st * C::kTileBytes, 16, 1024);
+        const uint64_t a = descQ0 + (uint64_t)(i * (C::kTileBytes >> 4));
+        const uint64_t b = descK0 + (uint64_t)(st * (C::kTileBytes >> 4));
         uint32_t acc = 0;
 #pragma unroll
-        for (int h = 0; h < C::kHalves; ++h) {
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4) {
-            mma_ss(d, a + 2 * k4, b + 2 * k4, kIdescQK, acc);          // 16 bf16 = 32 B = 2 descriptor units
-            acc = 1;
-          }
-          a += C::kPanelBytes >> 4;
-          b += C::kPanelBytes >> 4;
+        for (int kk = 0; kk < D / 16; ++kk) {
+          // 16 bf16 = 32 B = 2 descriptor units within a 64-column panel, panels kPanelBytes apart
+          const uint64_t off = (uint64_t)((kk >> 2) * (C::kPanelBytes >> 4) + (kk & 3) * 2);
+          mma_ss(d, a + off, b + off, kIdescQK, acc);
+          acc = 1;
         }
       };
       // O_i (+)= P_i[:, 16 kk .. 16 kk + 16) V[16 kk .. 16 kk + 16, :] for kk in [k0, k1); P_i is read from
       // the first 64 columns of S_i
       auto issue_pv = [&](int i, uint32_t st, int k0, int k1, uint32_t acc) {
         const uint32_t d = tmem_base + 256 + i * 128, a = tmem_base + i * 128;
-        uint64_t b = smem_desc_sw128(sKV + st * C::kTileBytes, C::kPanelBytes, 1024) + (uint64_t)(k0 * (2048 >> 4));
+        const uint64_t b = descV0 + (uint64_t)(st * (C::kTileBytes >> 4));
 #pragma unroll
         for (int kk = k0; kk < k1; ++kk) {
-          mma_ts(d, a + kk * 8, b, kIdescPV, acc);
+          mma_ts(d, a + kk * 8, b + (uint64_t)(kk * (2048 >> 4)), kIdescPV, acc);
           acc = 1;
-          b += 2048 >> 4;
         }
       };
       // Are the next `n` (1 or 2) stages of the ring filled?  Does not block (test_wait, not try_wait,
