@@ -31,7 +31,7 @@ ROUTE_BLOCKS = 1003 * 9          # the paper's evaluation volume: 1003 videos x 
 ROUTE_FRAMES = 12
 # DRAM bytes (read + write) of ONE attention launch, from an ncu capture of the kernel as it stands
 # (its summary is kept with the other profiler summaries); None for workloads that were not captured.
-ATTN_DRAM_BYTES_PER_LAUNCH = {"14b": 0.793e9}
+ATTN_DRAM_BYTES_PER_LAUNCH = {"14b": 0.759e9}
 CPU_SAMPLE_HEADS = 12           # heads of one step the CPU oracle is timed on (about 10-20 s of host work)
 
 
