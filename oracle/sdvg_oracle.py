@@ -3,7 +3,8 @@
 A plain, slow, fp64 NumPy statement of what the path computes: 3D-RoPE on q/k,
 block-causal attention of one block against the rolling KV cache, the ring
 commit with eviction, the worst-frame router with a forced rejection of block
-0, and the per-block speculative schedule that strings them together.  Nothing
+0, the per-block speculative schedule that strings them together, and the 8-bit
+(E4M3) variant of the cache and the attention.  Nothing
 here is blocked, fused or tuned; library matmul/exp are used as single steps.
 
 Only tests, the smoke check and the bench's ``cpu_baseline`` leg may import
@@ -250,11 +251,12 @@ class RingCacheRef:
     next_block and the slot map alone.  Contents are exact copies of the input.
     """
 
-    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int):
+    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int, dtype=np.uint16):
         if min(slots, heads, block_tokens, head_dim) <= 0:
             raise ValueError("bad cache shape")
         self.slots, self.heads, self.T, self.D = slots, heads, block_tokens, head_dim
-        self.k = np.zeros((slots, block_tokens, heads, head_dim), dtype=np.uint16)
+        self.dtype = np.dtype(dtype)          # uint16: bf16 bits; uint8: E4M3 codes
+        self.k = np.zeros((slots, block_tokens, heads, head_dim), dtype=self.dtype)
         self.v = np.zeros_like(self.k)
         self.next_block = 0
         self.slot_block = [-1] * slots
@@ -291,7 +293,7 @@ class RingCacheRef:
             ks.append(self.k[s])
             vs.append(self.v[s])
         if not ks:
-            e = np.zeros((0, self.heads, self.D), dtype=np.uint16)
+            e = np.zeros((0, self.heads, self.D), dtype=self.dtype)
             return e, e.copy()
         return np.concatenate(ks, axis=0), np.concatenate(vs, axis=0)
 
@@ -303,6 +305,87 @@ def block_attn_ref(q_bits, k_self_bits, v_self_bits, cache: RingCacheRef, block_
     k_all = np.concatenate([kw, k_self_bits], axis=0)
     v_all = np.concatenate([vw, v_self_bits], axis=0)
     return attn_ref(q_bits, k_all, v_all, scale, heads=heads, rows=rows)
+
+
+# --------------------------------------------------------------------------
+# 8-bit variant (Sec. 2 "Video generation": quantised attention kernels are named as orthogonal
+# speed-ups; the paper fixes no format, so this is the library's choice: OCP E4M3 codes with one
+# static scale per head, x ~ scale_h * decode(code))
+# --------------------------------------------------------------------------
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """E4M3 byte -> float64 from the format's definition: 1 sign, 4 exponent (bias 7), 3 mantissa bits;
+    exponent field 0 = subnormal (mantissa * 2^-9); no infinities; S.1111.111 is NaN; largest finite 448."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = c & 0x7
+    mag = np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * 2.0 ** (e.astype(np.float64) - 7.0))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return sign * mag
+
+
+def e4m3_encode(x) -> np.ndarray:
+    """Nearest E4M3 value, ties to the even code, magnitudes beyond 448 saturate to 448, NaN -> 0x7F.
+    One rounding from the exact input (the 127 non-negative finite values are searched directly)."""
+    x = np.asarray(x, dtype=np.float64)
+    grid = e4m3_decode(np.arange(0x7F, dtype=np.uint8))             # 0 .. 448, increasing with the code
+    a = np.minimum(np.abs(np.nan_to_num(x, nan=0.0)), 448.0)
+    hi = np.clip(np.searchsorted(grid, a, side="left"), 0, 0x7E)       # first code with value >= a
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = grid[hi] - a, a - grid[lo]
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(pick_hi, hi, lo).astype(np.uint8)
+    code = code | np.where(np.signbit(x), 0x80, 0).astype(np.uint8)
+    return np.where(np.isnan(x), np.uint8(0x7F), code).astype(np.uint8)
+
+
+def quant_e4m3_ref(x_bits: np.ndarray, inv_scale: np.ndarray) -> np.ndarray:
+    """bf16 [tokens, heads, dim] -> E4M3 codes: the element times its head's inverse scale as ONE fp32
+    multiplication (round to nearest), then the rounding of e4m3_encode."""
+    x = bf16_to_f32(x_bits)
+    inv = np.asarray(inv_scale, dtype=np.float32).reshape(1, -1, 1)
+    with np.errstate(over="ignore"):
+        y = (x * inv).astype(np.float32)
+    return e4m3_encode(y.astype(np.float64))
+
+
+def attn_e4m3_ref(q8: np.ndarray, k8: np.ndarray, v8: np.ndarray, qk_descale, v_descale, scale: float,
+                  heads=None, rows=None, row_chunk: int = 1024):
+    """Attention on dequantised operands, in fp64, nothing else rounded:
+      s_j = scale * qk_descale[h] * <dec(q_i), dec(k_j)>,  o = v_descale[h] * sum_j softmax(s)_j dec(v_j).
+    qk_descale[h] is the product of the q and k scales of head h, v_descale[h] the v scale.
+    Same conventions and return values as attn_ref."""
+    Tq, H, D = q8.shape
+    heads = list(range(H)) if heads is None else list(heads)
+    rows = np.arange(Tq) if rows is None else np.asarray(rows, dtype=np.int64)
+    qk_descale = np.asarray(qk_descale, dtype=np.float64)
+    v_descale = np.asarray(v_descale, dtype=np.float64)
+    o = np.empty((rows.size, len(heads), D), dtype=np.float64)
+    lse = np.empty((len(heads), rows.size), dtype=np.float64)
+    for hi, h in enumerate(heads):
+        kh = e4m3_decode(k8[:, h, :])
+        vh = e4m3_decode(v8[:, h, :])
+        for r0 in range(0, rows.size, row_chunk):
+            rr = rows[r0:r0 + row_chunk]
+            qh = e4m3_decode(q8[rr, h, :])
+            s = (qh @ kh.T) * (scale * qk_descale[h])
+            m = s.max(axis=1, keepdims=True)
+            p = np.exp(s - m)
+            l = p.sum(axis=1, keepdims=True)
+            o[r0:r0 + rr.size, hi, :] = (p @ vh) / l * v_descale[h]
+            lse[hi, r0:r0 + rr.size] = (m + np.log(l))[:, 0]
+    return o, lse
+
+
+def block_attn_e4m3_ref(q8, k_self8, v_self8, cache: "RingCacheRef", block_index: int, qk_descale, v_descale,
+                        scale: float, heads=None, rows=None):
+    """attn_e4m3_ref of block b against a ring of E4M3 codes (RingCacheRef with dtype uint8) and itself."""
+    kw, vw = cache.window(block_index)
+    k_all = np.concatenate([kw, k_self8], axis=0)
+    v_all = np.concatenate([vw, v_self8], axis=0)
+    return attn_e4m3_ref(q8, k_all, v_all, qk_descale, v_descale, scale, heads=heads, rows=rows)
 
 
 # --------------------------------------------------------------------------
