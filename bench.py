@@ -375,6 +375,30 @@ def run_ours(args):
         c3.close()
         del c2, c3, out2
 
+    # the 8-bit (E4M3) variant of the same attention: a secondary figure at reduced precision, never the headline
+    e4m3 = None
+    if args.workload != "tiny" and sh.head_dim == 128:
+        c8 = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device, e4m3=True)
+        inv = torch.full((sh.heads,), 448.0 / 4.5, device=device)      # static scales sized for 4.5 sigma of N(0, 1) data
+        desc = 1.0 / inv
+        for n in range(sh.slots - 1):
+            api.sdvg_kv_commit_e4m3(c8, st.k_r, st.v, inv, inv, n, api.SDVG_FINAL)
+        t_commit8 = time_call(lambda: api.sdvg_kv_commit_e4m3(c8, st.k_r, st.v, inv, inv, sh.slots - 1, api.SDVG_STAGE))
+        q8 = torch.empty(st.q_r.shape, dtype=torch.uint8, device=device)
+        api.sdvg_quant_e4m3(st.q_r, inv, q8)
+        t_attn8 = time_call(lambda: api.sdvg_block_attn_fwd_e4m3(q8, None, None, c8, sh.slots - 1, desc * desc, desc, st.out,
+                                                                 None, sh.scale, st.ws), n=40)
+        assert api.sdvg_block_attn_status(st.ws) == api.SDVG_OK
+        elems = sh.block_tokens * sh.heads * sh.head_dim
+        e4m3 = {"kernel": "sdvg_block_attn_fwd_e4m3", "ms": t_attn8, "tflops": attn_flops(sh, st.lk) / t_attn8 / 1e9,
+                "peak": 2 * pk["bf16_tflops"], "peak_source": "measured bf16 peak x the nominal fp8/bf16 ratio of 2",
+                "frac": attn_flops(sh, st.lk) / t_attn8 / 1e9 / (2 * pk["bf16_tflops"]),
+                "kv_commit_e4m3": {"ms": t_commit8, "gbs": 2 * elems * 3 / t_commit8 / 1e6,
+                                   "frac": 2 * elems * 3 / t_commit8 / 1e6 / pk["hbm_gbs"]},
+                "note": "operands E4M3 with one static scale per head, P rounded to E4M3; 40 launches back to back"}
+        c8.close()
+        del c8, q8
+
     # end to end through the same calls with host buffers: H2D of q,k,v,scores and D2H of out, accept per step,
     # copies of neighbouring steps overlapped with the kernels on separate streams
     st.e2e_setup()
@@ -434,6 +458,7 @@ def run_ours(args):
             "route": {"us": t_route * 1e3, "gbs": hb["route"] / t_route / 1e6}},
         "attention_by_fill_level": fill_levels,
         "attention_guidance_pair": pair,
+        "attention_e4m3": e4m3,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))

@@ -312,6 +312,61 @@ int sdvg_accept_stats(const uint8_t* accept, int num_blocks, int64_t first_block
  */
 int sdvg_state_copy(const void* const* src, void* const* dst, const size_t* bytes, int count, void* stream);
 
+/* ---- 8-bit (E4M3) variant of the cache and the attention --------------------- */
+/*
+ * Sec. 2 "Video generation" names quantised attention kernels as speed-ups orthogonal to the method and
+ * fixes no number format; this library's choice is the OCP E4M3 byte (1 sign, 4 exponent, 3 mantissa bits,
+ * bias 7, no infinities, largest finite value 448) with ONE STATIC SCALE PER HEAD and tensor:
+ * x ~ scale[head] * decode(code).  Every routine takes the INVERSE scales for quantising and the plain
+ * scales ("descale") for the attention; all scale arrays are device fp32 [heads], positive and finite.
+ * The bf16 path above stays the reference path; nothing here changes it.
+ */
+
+/*
+ * out[t, h, :] = e4m3(x[t, h, :] * inv_scale[h]): the product is one fp32 multiplication (round to nearest),
+ * the conversion rounds to nearest even and saturates at +-448 (NaN stays NaN, code 0x7F).
+ * x: device bf16 [tokens, heads, head_dim]; out: device bytes, same shape; head_dim 64 or 128.
+ * Used for q; k and v go through sdvg_kv_commit_e4m3.  Errors: INVALID_ARG, BAD_SHAPE, MISALIGNED.
+ */
+int sdvg_quant_e4m3(const void* x, const float* inv_scale, void* out, int tokens, int heads, int head_dim,
+                    void* stream);
+
+/* Bytes of ONE of the two buffers of an 8-bit ring (half of sdvg_cache_bytes); 0 unless head_dim is 128. */
+size_t sdvg_cache_bytes_e4m3(int slots, int heads, int block_tokens, int head_dim);
+
+/*
+ * As sdvg_cache_create, for a ring of E4M3 codes laid out [heads][slots][block_tokens][head_dim] bytes;
+ * head_dim must be 128.  The handle works with sdvg_cache_reset / _destroy / _state / _read_block (which
+ * then returns bytes), sdvg_kv_commit_e4m3 and sdvg_block_attn_fwd_e4m3; the bf16 entry points answer
+ * BAD_SHAPE for it, and the _e4m3 entry points answer BAD_SHAPE for a bf16 ring.
+ */
+int sdvg_cache_create_e4m3(sdvg_cache** out, void* k_buf, void* v_buf, int slots, int heads, int block_tokens,
+                           int head_dim);
+
+/*
+ * sdvg_kv_commit for an 8-bit ring: k_roped and v are device bf16 [block_tokens, heads, head_dim] and are
+ * quantised on the way into the slot as sdvg_quant_e4m3 does (k with k_inv_scale, v with v_inv_scale).
+ * Same ordering rules, flags, eviction report and errors as sdvg_kv_commit.
+ */
+int sdvg_kv_commit_e4m3(sdvg_cache* cache, const void* k_roped, const void* v, const float* k_inv_scale,
+                        const float* v_inv_scale, int64_t block_index, int flags, int64_t* evicted_block,
+                        void* stream);
+
+/*
+ * sdvg_block_attn_fwd on E4M3 operands:
+ *   out[i, h, :] = v_descale[h] * sum_j softmax_j(scale * qk_descale[h] * <dec q[i,h,:], dec K[j,h,:]>) dec V[j,h,:]
+ * with the same visible keys.  q8, k_self8, v_self8: device bytes [block_tokens, heads, 128] (k_self8 and
+ * v_self8 both NULL = the block was staged in the ring); cache: an 8-bit ring; qk_descale[h] = q scale * k
+ * scale of head h, v_descale[h] = v scale; out: device bf16; lse as in sdvg_block_attn_fwd (of the
+ * descaled logits).  Both products run on the tensor cores in E4M3 with fp32 accumulation; the softmax is
+ * fp32 and the probabilities are rounded to E4M3 (relative step 2^-4) before the second product, which is
+ * the one approximation beyond the operands' own quantisation.
+ * Errors: those of sdvg_block_attn_fwd; BAD_SHAPE for a bf16 ring.
+ */
+int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_self8, const sdvg_cache* cache,
+                             int64_t block_index, const float* qk_descale, const float* v_descale, void* out,
+                             float* lse, float scale, void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -60,6 +60,11 @@ SIGNATURES = {
     "sdvg_route_policy": (_I, [_VP, _VP, _I, _I, _I64, _I, _F, _I, _I, _I, _VP, _F, _VP, _VP, _VP, _VP]),
     "sdvg_accept_stats": (_I, [_VP, _I, _I64, _I, _VP, _VP]),
     "sdvg_state_copy": (_I, [_VP, _VP, _VP, _I, _VP]),
+    "sdvg_quant_e4m3": (_I, [_VP, _VP, _VP, _I, _I, _I, _VP]),
+    "sdvg_cache_bytes_e4m3": (_SZ, [_I, _I, _I, _I]),
+    "sdvg_cache_create_e4m3": (_I, [C.POINTER(_VP), _VP, _VP, _I, _I, _I, _I]),
+    "sdvg_kv_commit_e4m3": (_I, [_VP, _VP, _VP, _VP, _VP, _I64, _I, C.POINTER(_I64), _VP]),
+    "sdvg_block_attn_fwd_e4m3": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
 }
 
 _lib = None
@@ -152,19 +157,21 @@ def sdvg_rope3d_qk(q, k, q_out, k_out, grid, frame_offset: int, table: torch.Ten
 class Cache:
     """Rolling KV cache: torch owns the two device buffers, the library the ring state."""
 
-    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int, device="cuda"):
-        nbytes = lib().sdvg_cache_bytes(slots, heads, block_tokens, head_dim)
+    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int, device="cuda", e4m3: bool = False):
+        sizer = lib().sdvg_cache_bytes_e4m3 if e4m3 else lib().sdvg_cache_bytes
+        nbytes = sizer(slots, heads, block_tokens, head_dim)
         if nbytes == 0:
             raise SdvgError(SDVG_ERR_BAD_SHAPE, "sdvg_cache_bytes")
         self.slots, self.heads, self.block_tokens, self.head_dim = slots, heads, block_tokens, head_dim
+        self.e4m3 = e4m3                      # ring of E4M3 codes (8-bit variant) instead of bf16
         # physical layout [heads][slots][tokens][dim]; torch's allocator aligns to 512 B, so over-allocate
         self._k_raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
         self._v_raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
         self.k_ptr = (self._k_raw.data_ptr() + 1023) & ~1023
         self.v_ptr = (self._v_raw.data_ptr() + 1023) & ~1023
         h = _VP()
-        _check(lib().sdvg_cache_create(C.byref(h), self.k_ptr, self.v_ptr, slots, heads, block_tokens, head_dim),
-               "sdvg_cache_create")
+        create = lib().sdvg_cache_create_e4m3 if e4m3 else lib().sdvg_cache_create
+        _check(create(C.byref(h), self.k_ptr, self.v_ptr, slots, heads, block_tokens, head_dim), "sdvg_cache_create")
         self.handle = h
 
     def close(self):
@@ -191,7 +198,7 @@ class Cache:
     def read_block(self, slot: int, stream=None):
         """Logical [tokens, heads, dim] copies of the K and V held in ``slot``."""
         shape = (self.block_tokens, self.heads, self.head_dim)
-        k = torch.empty(shape, dtype=torch.bfloat16, device=self._k_raw.device)
+        k = torch.empty(shape, dtype=torch.uint8 if self.e4m3 else torch.bfloat16, device=self._k_raw.device)
         v = torch.empty_like(k)
         _check(lib().sdvg_cache_read_block(self.handle, slot, k.data_ptr(), v.data_ptr(), _stream(stream)),
                "sdvg_cache_read_block")
@@ -352,3 +359,52 @@ def sdvg_state_copy(srcs, dsts, stream=None) -> None:
                                C.cast((_VP * n)(*[_ptr(t) for t in dsts]), _VP),
                                C.cast((_SZ * n)(*nbytes), _VP), n, _stream(stream))
     _check(st, "sdvg_state_copy")
+
+
+# ---------------------------------------------------------------- 8-bit (E4M3) variant
+
+def _u8(t: Optional[torch.Tensor], shape=None):
+    if t is None:
+        return None
+    if t.dtype != torch.uint8:
+        raise ValueError("expected a uint8 tensor of E4M3 codes")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return _ptr(t)
+
+
+def _scales(t: torch.Tensor, heads: int):
+    if t.dtype != torch.float32 or tuple(t.shape) != (heads,):
+        raise ValueError("scales must be float32 [heads]")
+    return _ptr(t)
+
+
+def sdvg_quant_e4m3(x, inv_scale, out, stream=None) -> None:
+    tokens, heads, head_dim = x.shape
+    st = lib().sdvg_quant_e4m3(_bf16(x), _scales(inv_scale, heads), _u8(out, x.shape), tokens, heads, head_dim,
+                               _stream(stream))
+    _check(st, "sdvg_quant_e4m3")
+
+
+def sdvg_kv_commit_e4m3(cache: Cache, k_roped, v, k_inv_scale, v_inv_scale, block_index: int, flags: int,
+                        stream=None) -> int:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    ev = _I64(-1)
+    st = lib().sdvg_kv_commit_e4m3(cache.handle, _bf16(k_roped, shape), _bf16(v, shape),
+                                   _scales(k_inv_scale, cache.heads), _scales(v_inv_scale, cache.heads), block_index,
+                                   flags, C.byref(ev), _stream(stream))
+    _check(st, "sdvg_kv_commit_e4m3")
+    return ev.value
+
+
+def sdvg_block_attn_fwd_e4m3(q8, k_self8, v_self8, cache: Cache, block_index: int, qk_descale, v_descale, out, lse,
+                             scale: float, workspace: torch.Tensor, stream=None) -> None:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    if lse is not None and (lse.dtype != torch.float32 or tuple(lse.shape) != (cache.heads, cache.block_tokens)):
+        raise ValueError("lse must be float32 [heads, block_tokens]")
+    st = lib().sdvg_block_attn_fwd_e4m3(_u8(q8, shape), _u8(k_self8, None if k_self8 is None else shape),
+                                        _u8(v_self8, None if v_self8 is None else shape), cache.handle, block_index,
+                                        _scales(qk_descale, cache.heads), _scales(v_descale, cache.heads),
+                                        _bf16(out, shape), _ptr(lse), scale, workspace.data_ptr(), workspace.numel(),
+                                        _stream(stream))
+    _check(st, "sdvg_block_attn_fwd_e4m3")

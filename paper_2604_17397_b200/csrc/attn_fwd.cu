@@ -11,6 +11,9 @@
 // ends at the segment so that TMA zero-fills the ragged last tile; those columns are masked to
 // -inf before the row maximum.
 //
+// The 8-bit variant (sdvg_block_attn_fwd_e4m3) runs the same kernel template on E4M3 operands with per-head
+// scales; Sec. 2 names quantised attention as an orthogonal speed-up and fixes no format.
+//
 // Every wait on an mbarrier is bounded: kWaitLimitNs after kernel start a waiting thread gives up
 // and writes SDVG_ERR_TIMEOUT to the status word; all roles then fall through to the common exit,
 // which releases tensor memory.
@@ -55,6 +58,8 @@ struct alignas(64) AttnParams {
   int tokens, heads;
   float scale_log2e;                   // scale * log2(e): softmax is evaluated with exp2
   unsigned int* work;                  // [0] work counter, [1] status word
+  const float* qk_descale;             // 8-bit variant only: per head, q scale * k scale
+  const float* v_descale;              // 8-bit variant only: per head, v scale
 #ifdef SDVG_ATTN_DEBUG
   float* dbg;                          // S, P, O of the first key tile of CTA (0, 0)
 #endif
@@ -344,17 +349,17 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 matrix seen as (dim, rows, heads) with arbitrary row and head strides; box = 64 x 128 x 1,
-// 128-byte swizzle, rows beyond `rows` read as zero.
+// bf16 (elem_bytes 2) or byte (1) matrix seen as (dim, rows, heads) with arbitrary row and head strides;
+// box = 128 bytes x 128 rows x 1, 128-byte swizzle, rows beyond `rows` read as zero.
 int make_map(CUtensorMap* m, const void* base, int head_dim, long long rows, int heads, size_t row_stride_bytes,
-             size_t head_stride_bytes) {
+             size_t head_stride_bytes, int elem_bytes = 2) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return SDVG_ERR_CUDA;
   cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)rows, (cuuint64_t)heads};
   cuuint64_t strides[2] = {(cuuint64_t)row_stride_bytes, (cuuint64_t)head_stride_bytes};
-  cuuint32_t box[3] = {64, (cuuint32_t)kTileN, 1};
+  cuuint32_t box[3] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)kTileN, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = fn(m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SDVG_OK : SDVG_ERR_CUDA;
@@ -374,13 +379,13 @@ int launch_simple(const AttnParams& p, cudaStream_t stream) {
   return sdvg::cuda_status(cudaGetLastError());
 }
 
-template <int D>
+template <int D, bool F8 = false>
 int launch_ws(const AttnParams& p, cudaStream_t stream) {
   static bool configured = false;
   static int sms = 0;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         WsCfg<D>::kDynamic);
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         WsCfg<D, F8>::kDynamic);
     if (e != cudaSuccess) return sdvg::cuda_status(e);
     int dev = 0;
     cudaGetDevice(&dev);
@@ -389,7 +394,7 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
   }
   const int total_tiles = ((p.tokens + kTileM - 1) / kTileM) * p.heads * p.batch;
   const int grid = total_tiles < sms ? total_tiles : sms;
-  attn_fwd_ws_kernel<D><<<grid, WsCfg<D>::kThreads, WsCfg<D>::kDynamic, stream>>>(p);
+  attn_fwd_ws_kernel<D, F8><<<grid, WsCfg<D, F8>::kThreads, WsCfg<D, F8>::kDynamic, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
 }
 
@@ -420,12 +425,13 @@ int check_problem(const void* q, const void* k_self, const void* v_self, const s
 int fill_problem(AttnProblem& pr, int* seg_len, int* nseg_out, const void* q, const void* k_self, const void* v_self,
                  const sdvg_cache* c, int64_t block_index, void* out, float* lse) {
   const int T = c->block_tokens, H = c->heads, D = c->head_dim, S = c->slots;
-  const size_t row_bytes = (size_t)D * 2;
+  const int eb = c->elem_bytes;                      // q, k_self and v_self have the cache's element type
+  const size_t row_bytes = (size_t)D * eb;
   const size_t ring_head_stride = (size_t)S * T * row_bytes;
   int st, nseg = 0;
   pr.out = (__nv_bfloat16*)out;
   pr.lse = lse;
-  if ((st = make_map(&pr.q_map, q, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+  if ((st = make_map(&pr.q_map, q, D, T, H, (size_t)H * row_bytes, row_bytes, eb)) != SDVG_OK) return st;
 
   // Visible committed blocks: the last S-1 before block_index, living in slots (b % S).  Their slots
   // form at most two runs of consecutive slots; with the block staged, its slot joins them.
@@ -447,15 +453,15 @@ int fill_problem(AttnProblem& pr, int* seg_len, int* nseg_out, const void* q, co
     const long long rows = (long long)(e - s) * T;
     const char* kb = (const char*)c->k_buf + (size_t)s * T * row_bytes;
     const char* vb = (const char*)c->v_buf + (size_t)s * T * row_bytes;
-    if ((st = make_map(&pr.k_map[nseg], kb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
-    if ((st = make_map(&pr.v_map[nseg], vb, D, rows, H, row_bytes, ring_head_stride)) != SDVG_OK) return st;
+    if ((st = make_map(&pr.k_map[nseg], kb, D, rows, H, row_bytes, ring_head_stride, eb)) != SDVG_OK) return st;
+    if ((st = make_map(&pr.v_map[nseg], vb, D, rows, H, row_bytes, ring_head_stride, eb)) != SDVG_OK) return st;
     seg_len[nseg++] = (int)rows;
     s = e;
   }
   if (k_self) {
     if (nseg >= kMaxSegments) return SDVG_ERR_BAD_STATE;
-    if ((st = make_map(&pr.k_map[nseg], k_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
-    if ((st = make_map(&pr.v_map[nseg], v_self, D, T, H, (size_t)H * row_bytes, row_bytes)) != SDVG_OK) return st;
+    if ((st = make_map(&pr.k_map[nseg], k_self, D, T, H, (size_t)H * row_bytes, row_bytes, eb)) != SDVG_OK) return st;
+    if ((st = make_map(&pr.v_map[nseg], v_self, D, T, H, (size_t)H * row_bytes, row_bytes, eb)) != SDVG_OK) return st;
     seg_len[nseg++] = T;
   }
   *nseg_out = nseg;
@@ -466,8 +472,10 @@ int fill_problem(AttnProblem& pr, int* seg_len, int* nseg_out, const void* q, co
 // problems of one shape, fused into one launch when their key segments agree, else launched one by one.
 int attn_forward_batch(int batch, const void* const* q, const void* const* k_self, const void* const* v_self,
                        const sdvg_cache* const* caches, const int64_t* block_index, void* const* out,
-                       float* const* lse, float scale, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+                       float* const* lse, float scale, void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                       int elem_bytes = 2, const float* qk_descale = nullptr, const float* v_descale = nullptr) {
   if (batch < 1 || !q || !caches || !block_index || !out || !workspace) return SDVG_ERR_INVALID_ARG;
+  if (elem_bytes == 1 && (batch != 1 || !qk_descale || !v_descale)) return SDVG_ERR_INVALID_ARG;
   if (batch > kMaxBatch) return SDVG_ERR_BAD_SHAPE;
   if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
   if (!(scale > 0.f) || !isfinite(scale)) return SDVG_ERR_INVALID_ARG;
@@ -475,7 +483,7 @@ int attn_forward_batch(int batch, const void* const* q, const void* const* k_sel
   for (int b = 0; b < batch; ++b) {
     if (!caches[b]) return SDVG_ERR_INVALID_ARG;
     if (caches[b]->block_tokens != caches[0]->block_tokens || caches[b]->heads != caches[0]->heads ||
-        caches[b]->head_dim != caches[0]->head_dim)
+        caches[b]->head_dim != caches[0]->head_dim || caches[b]->elem_bytes != elem_bytes)
       return SDVG_ERR_BAD_SHAPE;
   }
   int st;
@@ -490,6 +498,8 @@ int attn_forward_batch(int batch, const void* const* q, const void* const* k_sel
   p.heads = caches[0]->heads;
   p.scale_log2e = scale * 1.4426950408889634f;
   p.work = (unsigned int*)workspace;
+  p.qk_descale = qk_descale;
+  p.v_descale = v_descale;
   const int D = caches[0]->head_dim;
   bool same = true;
   int seg_len[kMaxBatch][kMaxSegments] = {}, nseg[kMaxBatch] = {};
@@ -508,6 +518,7 @@ int attn_forward_batch(int batch, const void* const* q, const void* const* k_sel
   cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
   if (e != cudaSuccess) return sdvg::cuda_status(e);
   auto launch = [&](const AttnParams& pp) {
+    if (elem_bytes == 1) return launch_ws<128, true>(pp, stream);     // an 8-bit cache always has head_dim 128
     if (use_simple_kernel()) return D == 128 ? launch_simple<128>(pp, stream) : launch_simple<64>(pp, stream);
     return D == 128 ? launch_ws<128>(pp, stream) : launch_ws<64>(pp, stream);
   };
@@ -579,6 +590,20 @@ int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* con
                                 void* workspace, size_t workspace_bytes, void* stream_) {
   return attn_forward_batch(batch, q, k_self, v_self, caches, block_index, out, lse, scale, workspace,
                             workspace_bytes, (cudaStream_t)stream_);
+}
+
+int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_self8, const sdvg_cache* c,
+                             int64_t block_index, const float* qk_descale, const float* v_descale, void* out,
+                             float* lse, float scale, void* workspace, size_t workspace_bytes, void* stream_) {
+  if (!c || !qk_descale || !v_descale) return SDVG_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(qk_descale) | reinterpret_cast<uintptr_t>(v_descale)) & 3) return SDVG_ERR_MISALIGNED;
+  const void* const qs[1] = {q8};
+  const void* const ks[1] = {k_self8};
+  const void* const vs[1] = {v_self8};
+  void* const outs[1] = {out};
+  float* const lses[1] = {lse};
+  return attn_forward_batch(1, qs, k_self8 ? ks : nullptr, v_self8 ? vs : nullptr, &c, &block_index, outs, lses, scale,
+                            workspace, workspace_bytes, (cudaStream_t)stream_, 1, qk_descale, v_descale);
 }
 
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,

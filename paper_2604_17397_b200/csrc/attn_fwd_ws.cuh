@@ -37,6 +37,12 @@
 // [0, 1) plus a cubic, relative error 2e-4, a tenth of the bf16 rounding P gets anyway); it is off by
 // default (SDVG_ATTN_POLY_PAIRS = 0) because the extra instructions cost more than the freed
 // special-function slots gain once the GPU runs under its power cap.
+//
+// 8-bit variant (template flag F8): Q, K and V tiles are E4M3 bytes (a 128-dim row is one 128-byte panel, so a
+// tile is half the size and the ring holds 8 stages), both products use the 8-bit MMA kind (K = 32 per
+// instruction, half the tensor-pipe time), P is rounded to E4M3 (four per TMEM column) and the per-head
+// scales enter as a factor of the logit scale and of the final 1/l.  Everything else (roles, barriers,
+// schedule, lazy maximum, split tiles) is shared; the softmax, not the tensor pipe, then sets the pace.
 #pragma once
 
 #ifdef SDVG_ATTN_TRACE
@@ -60,12 +66,15 @@ __device__ long long* g_trace = nullptr;     // [6 roles][512 events][id, clock]
 #define SDVG_TRACE(role, id) do { } while (0)
 #endif
 
-template <int D>
+// F8: operands are E4M3 bytes instead of bf16 (a row of 128 dims is then one 128-byte panel).
+template <int D, bool F8 = false>
 struct WsCfg {
-  static constexpr int kHalves = D / 64;
+  static_assert(!F8 || D == 128, "the 8-bit variant is built for head_dim 128");
+  static constexpr int kHalves = F8 ? D / 128 : D / 64;             // 128-byte panels per row
   static constexpr int kPanelBytes = 128 * 128;
   static constexpr int kTileBytes = kHalves * kPanelBytes;          // one Q, K or V tile
-  static constexpr int kStages = (D == 128) ? 5 : 8;                // K/V ring entries (K and V alternate)
+  static constexpr int kStages = (D == 128 && !F8) ? 5 : 8;         // K/V ring entries (K and V alternate)
+  static constexpr int kPanelElems = F8 ? 128 : 64;                 // elements per panel row
   static constexpr int kQ = 0;                                      // two query tiles
   static constexpr int kKV = 2 * kTileBytes;
   static constexpr int kRowState = kKV + kStages * kTileBytes;      // float [2][128]: -m*c2 of a row, later the helper's l
@@ -209,6 +218,10 @@ __device__ __forceinline__ void exp2_poly2(uint64_t x2, float& e0, float& e1) {
 #define SDVG_ATTN_POLY_PAIRS 0
 #endif
 
+#ifndef SDVG_ATTN_POLY_PAIRS_F8
+#define SDVG_ATTN_POLY_PAIRS_F8 0
+#endif
+
 // One 32-column chunk of a row: P = 2^(c2 * S - m*c2) as bf16 pairs, returns the packed partial row sums.
 __device__ __forceinline__ void exp_chunk(const uint32_t (&s)[32], uint64_t c2x2, uint64_t negx2, uint32_t (&pk)[16],
                                           uint64_t& sum_a, uint64_t& sum_b) {
@@ -231,6 +244,41 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&s)[32], uint64_t c2x2
   }
 }
 
+// The same chunk as E4M3 bytes (four per word); the row sums are taken before the rounding, as above.
+__device__ __forceinline__ void exp_chunk_f8(const uint32_t (&s)[32], uint64_t c2x2, uint64_t negx2, uint32_t (&pk)[8],
+                                             uint64_t& sum_a, uint64_t& sum_b) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    float e[4];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const uint64_t x2 =
+          fma2(pack2(__uint_as_float(s[4 * k + 2 * u]), __uint_as_float(s[4 * k + 2 * u + 1])), c2x2, negx2);
+      if (((2 * k + u) & 3) < SDVG_ATTN_POLY_PAIRS_F8) {
+        exp2_poly2(x2, e[2 * u], e[2 * u + 1]);
+      } else {
+        float x0, x1;
+        unpack2(x2, x0, x1);
+        e[2 * u] = fast_exp2(x0);
+        e[2 * u + 1] = fast_exp2(x1);
+      }
+    }
+    sum_a = add2(sum_a, pack2(e[0], e[1]));
+    sum_b = add2(sum_b, pack2(e[2], e[3]));
+    pk[k] = pack_e4m3x4(e[0], e[1], e[2], e[3]);
+  }
+}
+
+// Reference-maximum policy.  P = 2^(c2 S - m_ref c2 + shift) and the reference is only raised when the row
+// maximum outgrew it by more than `lazy` (in the exp2 domain), so P <= 2^(shift + lazy).  bf16 has the
+// range for 2^8; E4M3 ends at 448, and its precision ends 2^-9 below 1, so there the window is moved up:
+// P <= 2^8 still, and a key 2^-12 below the reference still gets a normal number.
+template <bool F8>
+struct RefMax {
+  static constexpr float kLazy = F8 ? 4.f : 8.f;
+  static constexpr float kShift = F8 ? 4.f : 0.f;
+};
+
 __device__ __forceinline__ void max_chunk(const uint32_t (&s)[32], float (&mx)[4]) {
 #pragma unroll
   for (int k = 0; k < 32; k += 8)
@@ -239,9 +287,9 @@ __device__ __forceinline__ void max_chunk(const uint32_t (&s)[32], float (&mx)[4
       mx[u] = fmax3(mx[u], __uint_as_float(s[k + 2 * u]), __uint_as_float(s[k + 2 * u + 1]));
 }
 
-template <int D>
+template <int D, bool F8 = false>
 __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_constant__ AttnParams p) {
-  using C = WsCfg<D>;
+  using C = WsCfg<D, F8>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   // [2][128]: while an item runs, -m_ref * c2 of the row (softmax -> helper); at its end the helper's
@@ -334,7 +382,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           const CUtensorMap* m = is_v ? &pr.v_map[seg] : &pr.k_map[seg];
           for (int h = 0; h < C::kHalves; ++h)
             tma_load_3d(smem + C::kKV + ring.stage * C::kTileBytes + h * C::kPanelBytes, m, &kv_full[ring.stage],
-                        h * 64, kt * kTileN, head % p.heads);
+                        h * C::kPanelElems, kt * kTileN, head % p.heads);
         }
         ring.template advance<C::kStages>();
         ++kv_issued;
@@ -353,7 +401,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             mbar_expect_tx(&q_full[i], C::kTileBytes);
             for (int h = 0; h < C::kHalves; ++h)
               tma_load_3d(smem + C::kQ + i * C::kTileBytes + h * C::kPanelBytes, &p.prob[it.head[i] / p.heads].q_map,
-                          &q_full[i], h * 64, it.tile[i] * kTileM, it.head[i] % p.heads);
+                          &q_full[i], h * C::kPanelElems, it.tile[i] * kTileM, it.head[i] % p.heads);
           }
         }
         // K/V tiles in the order the issuer consumes them: K of the first key tile of every stream, then
@@ -377,8 +425,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     } else if (warp == 13) {
       // ---- MMA issuer ---------------------------------------------------------------------
       const bool leader = elect_one();
-      constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, false);
-      constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, true);
+      constexpr uint32_t kIdescQK = F8 ? idesc_e4m3_f32(kTileM, kTileN, false) : idesc_bf16_f32(kTileM, kTileN, false);
+      constexpr uint32_t kIdescPV = F8 ? idesc_e4m3_f32(kTileM, D, true) : idesc_bf16_f32(kTileM, D, true);
       const uint32_t sQ = smem_u32(smem + C::kQ), sKV = smem_u32(smem + C::kKV);
       uint32_t q_cnt[2] = {0, 0};
       uint32_t pv_par = 0;                 // bit i: phase parity of lane i's P barriers
@@ -402,9 +450,11 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         uint32_t acc = 0;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          // 16 bf16 = 32 B = 2 descriptor units within a 64-column panel, panels kPanelBytes apart
+          if (F8 && kk >= D / 32) break;                   // an 8-bit MMA covers 32 dims
+          // one MMA reads 32 B of every row = 2 descriptor units within a 128-byte panel, panels kPanelBytes apart
           const uint64_t off = (uint64_t)((kk >> 2) * (C::kPanelBytes >> 4) + (kk & 3) * 2);
-          mma_ss(d, a + off, b + off, kIdescQK, acc);
+          if constexpr (F8) mma_ss_f8(d, a + off, b + off, kIdescQK, acc);
+          else mma_ss(d, a + off, b + off, kIdescQK, acc);
           acc = 1;
         }
       };
@@ -415,10 +465,14 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         const uint64_t b = descV0 + (uint64_t)(st * (C::kTileBytes >> 4));
 #pragma unroll
         for (int kk = k0; kk < k1; ++kk) {
-          mma_ts(d, a + kk * 8, b + (uint64_t)(kk * (2048 >> 4)), kIdescPV, acc);
+          // slice kk of P is 8 TMEM columns (16 bf16 or 32 bytes per row); its keys are 16 or 32 rows of V
+          if constexpr (F8) mma_ts_f8(d, a + kk * 8, b + (uint64_t)(kk * (4096 >> 4)), kIdescPV, acc);
+          else mma_ts(d, a + kk * 8, b + (uint64_t)(kk * (2048 >> 4)), kIdescPV, acc);
           acc = 1;
         }
       };
+      // slices of P per 32-column chunk of S: chunk c of the softmax is slices [c kPc, c kPc + kPc)
+      constexpr int kPc = F8 ? 1 : 2;
       // Are the next `n` (1 or 2) stages of the ring filled?  Does not block (test_wait, not try_wait,
       // which may suspend the thread for microseconds when the answer is no).
       auto stages_filled = [&](int n) {
@@ -511,8 +565,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             SDVG_TRACE(2, 3000 + i * 1000 + t);
             tc_fence_after();
             if (leader) {
-              issue_pv(i, stV, 6, 8, t > 0 ? 1u : 0u);
-              issue_pv(i, stV, 0, 4, 1u);
+              issue_pv(i, stV, 3 * kPc, 4 * kPc, t > 0 ? 1u : 0u);
+              issue_pv(i, stV, 0, 2 * kPc, 1u);
             }
             // six MMAs are queued: take the stages of the next step that has stages of its own
             {
@@ -524,7 +578,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
             SDVG_TRACE(2, 5000 + i * 1000 + t);
             tc_fence_after();
             if (leader) {
-              issue_pv(i, stV, 4, 6, 1u);
+              issue_pv(i, stV, 2 * kPc, 3 * kPc, 1u);
               mma_commit(&o_full[i]);
               if (last_user) mma_commit(&kv_empty[stV]);
               if (more) {
@@ -549,6 +603,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     const uint32_t tO[2] = {tmem_base + 256 + lane_off, tmem_base + 384 + lane_off};
     const float c2 = p.scale_log2e;
     const uint64_t c2x2 = pack2(c2, c2);
+    uint64_t c2h[2] = {c2x2, c2x2};      // 8-bit variant: the logit scale carries the head's q and k scales
     uint32_t cnt[2] = {0, 0};            // (item, key tile) steps done per lane = phase index of its barriers
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && tid == 256)
@@ -557,6 +612,13 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       WsItem it;
       sched.get(v, ntiles_k, it);
       float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
+      if constexpr (F8) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const float c = c2 * __ldg(p.qk_descale + it.head[i]);
+          c2h[i] = pack2(c, c);
+        }
+      }
       #pragma unroll 1
       for (int j = 0; j < it.nk[0] && alive; ++j) {          // step j of lane i: that lane's j-th key tile
 #pragma unroll
@@ -591,12 +653,19 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           SDVG_TRACE(3, 20000 + 1000 * i + j);
           // ---- this row's share of P: key columns 96-127 -------------------------------------
           tc_fence_after();
-          uint32_t s3[32], pk[16];
+          uint32_t s3[32];
           tmem_ld32(tS[i] + 96, s3);
           tmem_wait_ld();
           uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-          exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
-          tmem_st16(tS[i] + 48, pk);
+          if constexpr (F8) {
+            uint32_t pk[8];
+            exp_chunk_f8(s3, c2h[i], pack2(neg, neg), pk, sum_a, sum_b);
+            tmem_st8(tS[i] + 24, pk);
+          } else {
+            uint32_t pk[16];
+            exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
+            tmem_st16(tS[i] + 48, pk);
+          }
           {
             float a0, a1, b0, b1;
             unpack2(sum_a, a0, a1);
@@ -627,8 +696,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem_base + i * 128 + lane_off;
     const uint32_t tO = tmem_base + 256 + i * 128 + lane_off;
-    const float c2 = p.scale_log2e;
-    const uint64_t c2x2 = pack2(c2, c2);
+    float c2 = p.scale_log2e;
+    uint64_t c2x2 = pack2(c2, c2);
     uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0, split_cnt = 0;
     bool alive = true;
     SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0)
@@ -641,7 +710,11 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       const int my_nk = i == 0 ? it.nk[0] : it.nk[1];
       const int my_tile = i == 0 ? it.tile[0] : it.tile[1];
       const int my_head = i == 0 ? it.head[0] : it.head[1];
-      float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2
+      if constexpr (F8) {                                  // the logit scale carries the head's q and k scales
+        c2 = p.scale_log2e * __ldg(p.qk_descale + my_head);
+        c2x2 = pack2(c2, c2);
+      }
+      float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2 (+ the window shift)
       {
         #pragma unroll 1
         for (int j = 0; j < my_nk && alive; ++j) {        // this lane's j-th key tile
@@ -691,9 +764,9 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           const float mxa = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
           if (j == 0) {
             m_ref = mxa;
-            neg = __fmul_rn(-mxa, c2);
-          } else if ((mxa - m_ref) * c2 > 8.f) {
-            const float neg_new = __fmul_rn(-mxa, c2);
+            neg = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
+          } else if ((mxa - m_ref) * c2 > RefMax<F8>::kLazy) {
+            const float neg_new = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
             l_run *= fast_exp2(__fsub_rn(neg_new, neg));      // the helper derives the same factor from the same two values
             m_ref = mxa;
             neg = neg_new;
@@ -704,17 +777,29 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           // ---- P = 2^(c2 * (S - m_ref)), bf16, written back over S: columns 0-63, then 64-95 ------
           const uint64_t negx2 = pack2(neg, neg);
           uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-          uint32_t pk[16];
-          exp_chunk(s[0], c2x2, negx2, pk, sum_a, sum_b);
-          tmem_st16(tS, pk);
-          exp_chunk(s[1], c2x2, negx2, pk, sum_a, sum_b);
-          tmem_st16(tS + 16, pk);
+          uint32_t pk[F8 ? 8 : 16];
+          if constexpr (F8) {
+            exp_chunk_f8(s[0], c2x2, negx2, pk, sum_a, sum_b);
+            tmem_st8(tS, pk);
+            exp_chunk_f8(s[1], c2x2, negx2, pk, sum_a, sum_b);
+            tmem_st8(tS + 8, pk);
+          } else {
+            exp_chunk(s[0], c2x2, negx2, pk, sum_a, sum_b);
+            tmem_st16(tS, pk);
+            exp_chunk(s[1], c2x2, negx2, pk, sum_a, sum_b);
+            tmem_st16(tS + 16, pk);
+          }
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(&p_lo[i]);
           SDVG_TRACE(i, 4000 + j);
-          exp_chunk(s[2], c2x2, negx2, pk, sum_a, sum_b);
-          tmem_st16(tS + 32, pk);
+          if constexpr (F8) {
+            exp_chunk_f8(s[2], c2x2, negx2, pk, sum_a, sum_b);
+            tmem_st8(tS + 16, pk);
+          } else {
+            exp_chunk(s[2], c2x2, negx2, pk, sum_a, sum_b);
+            tmem_st16(tS + 32, pk);
+          }
           {
             float a0, a1, b0, b1;
             unpack2(sum_a, a0, a1);
@@ -764,7 +849,7 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       const int grow = my_tile * kTileM + row;
       const AttnProblem& pr = p.prob[my_head / p.heads];
       const int head = my_head % p.heads;
-      const float inv = 1.f / l_run;
+      const float inv = F8 ? __ldg(p.v_descale + head) / l_run : 1.f / l_run;     // 8-bit: V's scale of this head
       w0 *= inv;
       w1 *= inv;
 #pragma unroll 1

@@ -185,6 +185,7 @@ int sdvg_rope3d_qk(const void* q, const void* k, void* q_out, void* k_out, int t
 int sdvg_kv_commit(sdvg_cache* c, const void* k_roped, const void* v, int64_t block_index, int flags,
                    int64_t* evicted_block, void* stream) {
   if (!c || !k_roped || !v) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 2) return SDVG_ERR_BAD_SHAPE;          // an 8-bit cache takes sdvg_kv_commit_e4m3
   if (!sdvg::aligned16(k_roped) || !sdvg::aligned16(v)) return SDVG_ERR_MISALIGNED;
   int slot = 0;
   int st = sdvg::ring_begin_commit(c, block_index, flags, &slot);
@@ -209,6 +210,7 @@ int sdvg_rope3d_qk_commit(sdvg_cache* c, const void* q, const void* k, const voi
                           const float* cos_sin_tab, int tab_frames, int64_t block_index, int flags,
                           int64_t* evicted_block, void* stream) {
   if (!c || !k || !v) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 2) return SDVG_ERR_BAD_SHAPE;
   if ((q == nullptr) != (q_out == nullptr)) return SDVG_ERR_INVALID_ARG;
   if (!sdvg::aligned16(q) || !sdvg::aligned16(k) || !sdvg::aligned16(v) || !sdvg::aligned16(q_out) ||
       !sdvg::aligned16(k_out))
@@ -240,16 +242,17 @@ int sdvg_cache_read_block(const sdvg_cache* c, int slot, void* k_out, void* v_ou
   if (!sdvg::aligned16(k_out) || !sdvg::aligned16(v_out)) return SDVG_ERR_MISALIGNED;
   int st = sdvg::require_sm100();
   if (st != SDVG_OK) return st;
-  const long long stride = (long long)c->slots * c->block_tokens * (c->head_dim / 8);
-  const long long total = (long long)c->block_tokens * c->heads * (c->head_dim / 8);
+  const int vpr = c->head_dim * c->elem_bytes / 16;          // 16-byte vectors per (token, head) row: 16 or 8
+  const long long stride = (long long)c->slots * c->block_tokens * vpr;
+  const long long total = (long long)c->block_tokens * c->heads * vpr;
   const unsigned blocks = (unsigned)((total + kThreads - 1) / kThreads < 148 * 8 ? (total + kThreads - 1) / kThreads
                                                                                   : 148 * 8);
   const void* bufs[2] = {c->k_buf, c->v_buf};
   void* outs[2] = {k_out, v_out};
   for (int i = 0; i < 2; ++i) {
     if (!outs[i]) continue;
-    const uint4* base = (const uint4*)bufs[i] + sdvg::slot_offset(c, 0, slot) / 8;
-    if (c->head_dim == 128)
+    const uint4* base = (const uint4*)bufs[i] + sdvg::slot_offset(c, 0, slot) * c->elem_bytes / 16;
+    if (vpr == 16)
       slot_read_kernel<128><<<blocks, kThreads, 0, (cudaStream_t)stream>>>(base, (uint4*)outs[i], c->block_tokens,
                                                                           c->heads, stride);
     else

@@ -136,11 +136,26 @@ int sdvg_cache_create(sdvg_cache** out, void* k_buf, void* v_buf, int slots, int
   c->heads = heads;
   c->block_tokens = block_tokens;
   c->head_dim = head_dim;
+  c->elem_bytes = 2;
   c->next_block = 0;
   c->staged_block = -1;
   c->slot_block.assign(slots, -1);
   *out = c;
   return SDVG_OK;
+}
+
+size_t sdvg_cache_bytes_e4m3(int slots, int heads, int block_tokens, int head_dim) {
+  if (head_dim != 128) return 0;
+  return sdvg_cache_bytes(slots, heads, block_tokens, head_dim) / 2;
+}
+
+int sdvg_cache_create_e4m3(sdvg_cache** out, void* k_buf, void* v_buf, int slots, int heads, int block_tokens,
+                           int head_dim) {
+  if (slots > 0 && heads > 0 && block_tokens > 0 && sdvg::head_dim_ok(head_dim) && head_dim != 128)
+    return SDVG_ERR_BAD_SHAPE;
+  const int st = sdvg_cache_create(out, k_buf, v_buf, slots, heads, block_tokens, head_dim);
+  if (st == SDVG_OK) (*out)->elem_bytes = 1;
+  return st;
 }
 
 int sdvg_cache_reset(sdvg_cache* c) {

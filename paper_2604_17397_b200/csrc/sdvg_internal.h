@@ -12,6 +12,7 @@ struct sdvg_cache {
   void* k_buf;
   void* v_buf;
   int slots, heads, block_tokens, head_dim;
+  int elem_bytes;                       // 2: bf16 elements; 1: E4M3 codes (8-bit variant)
   int64_t next_block;
   int64_t staged_block;                 // block whose provisional K/V sit in its slot, -1 if none
   std::vector<int64_t> slot_block;      // slot -> committed block, -1 = empty
@@ -29,7 +30,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline bool head_dim_ok(int d) { return d == 64 || d == 128; }
 
-// Element offset of (head, slot, token 0, dim 0) in a cache buffer laid out [heads][slots][tokens][dim].
+// Element (not byte) offset of (head, slot, token 0, dim 0) in a cache buffer laid out [heads][slots][tokens][dim].
 inline size_t slot_offset(const sdvg_cache* c, int head, int slot) {
   return ((size_t)head * c->slots + slot) * (size_t)c->block_tokens * c->head_dim;
 }

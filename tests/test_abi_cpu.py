@@ -107,3 +107,40 @@ def test_rope_and_route_argument_checks(lib):
     assert t(0x1000, None, 0, 12, 0, -0.7, 0x2000, 0x3000, None, None) == api.SDVG_OK      # nothing to do
     assert t(None, None, 4, 12, 0, -0.7, 0x2000, 0x3000, None, None) == api.SDVG_ERR_INVALID_ARG
     assert t(0x1002, None, 4, 12, 0, -0.7, 0x2000, 0x3000, None, None) == api.SDVG_ERR_MISALIGNED
+
+
+def test_e4m3_entry_points_validate_on_the_host(lib):
+    assert lib.sdvg_cache_bytes_e4m3(7, 40, 4680, 128) == 7 * 40 * 4680 * 128
+    assert lib.sdvg_cache_bytes_e4m3(7, 40, 4680, 64) == 0
+    h8, h16 = C.c_void_p(), C.c_void_p()
+    assert lib.sdvg_cache_create_e4m3(C.byref(h8), 0x10000, 0x20000, 3, 2, 64, 64) == api.SDVG_ERR_BAD_SHAPE
+    assert lib.sdvg_cache_create_e4m3(C.byref(h8), 0x10010, 0x20000, 3, 2, 64, 128) == api.SDVG_ERR_MISALIGNED
+    assert lib.sdvg_cache_create_e4m3(C.byref(h8), 0x10000, 0x20000, 3, 2, 64, 128) == api.SDVG_OK
+    assert lib.sdvg_cache_create(C.byref(h16), 0x10000, 0x20000, 3, 2, 64, 128) == api.SDVG_OK
+    sc = 0x90000
+    commit8 = lib.sdvg_kv_commit_e4m3
+    # the element types of ring and entry point must agree, either way round
+    assert commit8(h16, 0x30000, 0x40000, sc, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert lib.sdvg_kv_commit(h8, 0x30000, 0x40000, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert lib.sdvg_rope3d_qk_commit(h8, None, 0x30000, 0x40000, None, None, 1, 8, 8, 0, 0x80000, 4, 0, api.SDVG_FINAL,
+                                     None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert commit8(h8, 0x30000, 0x40000, sc, sc, 1, api.SDVG_FINAL, None, None) == api.SDVG_ERR_BAD_STATE
+    assert commit8(h8, 0x30000, 0x40000, sc, sc, 0, 3, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert commit8(h8, 0x30000, 0x40000, None, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert commit8(h8, 0x30008, 0x40000, sc, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_MISALIGNED
+    assert commit8(h8, 0x30000, 0x40000, sc + 2, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_MISALIGNED
+    ws = lib.sdvg_block_attn_workspace_bytes()
+    f8, f16 = lib.sdvg_block_attn_fwd_e4m3, lib.sdvg_block_attn_fwd
+    assert f8(0x50000, 0x30000, 0x40000, h16, 0, sc, sc, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_SHAPE
+    assert f16(0x50000, 0x30000, 0x40000, h8, 0, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_SHAPE
+    assert f8(0x50000, None, None, h8, 0, sc, sc, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_STATE
+    assert f8(0x50000, 0x30000, 0x40000, h8, 1, sc, sc, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_STATE
+    assert f8(0x50000, 0x30000, 0x40000, h8, 0, None, sc, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_INVALID_ARG
+    assert f8(0x50000, 0x30000, 0x40000, h8, 0, sc, sc + 1, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_MISALIGNED
+    assert f8(0x50000, 0x30000, 0x40000, h8, 0, sc, sc, 0x60000, None, 0.125, 0x70000, 4, None) == api.SDVG_ERR_INVALID_ARG
+    q = lib.sdvg_quant_e4m3
+    assert q(0x1000, sc, 0x2000, 16, 2, 96, None) == api.SDVG_ERR_BAD_SHAPE
+    assert q(0x1000, sc, 0x2000, 0, 2, 128, None) == api.SDVG_ERR_BAD_SHAPE
+    assert q(0x1000, None, 0x2000, 16, 2, 128, None) == api.SDVG_ERR_INVALID_ARG
+    assert q(0x1008, sc, 0x2000, 16, 2, 128, None) == api.SDVG_ERR_MISALIGNED
+    assert lib.sdvg_cache_destroy(h8) == 0 and lib.sdvg_cache_destroy(h16) == 0
