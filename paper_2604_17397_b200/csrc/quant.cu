@@ -56,7 +56,7 @@ int launch(const QuantParams& p, int njobs, cudaStream_t stream) {
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   long long want = (total + kThreads - 1) / kThreads;
-  long long cap = (long long)sms * 8 / njobs;                 // whole waves of 8 resident blocks per SM
+  long long cap = (long long)sms * 32 / njobs;                // few passes per thread; bounds the grid for very large tensors
   if (cap < 1) cap = 1;
   dim3 grid((unsigned)(want < cap ? want : cap), njobs, 1);
   quant_e4m3_kernel<<<grid, kThreads, 0, stream>>>(p);

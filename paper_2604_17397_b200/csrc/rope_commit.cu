@@ -150,10 +150,12 @@ int launch(RopeCommitParams& p, int head_dim, cudaStream_t stream) {
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int groups = (p.heads + kHeadGroup - 1) / kHeadGroup;
   long long want = (total + kThreads - 1) / kThreads;
-  // a whole number of waves: up to 8 resident 256-thread blocks per SM shared by the (y, z) slices
-  long long cap = (long long)sms * 8 / (groups * p.njobs);
+  // Enough blocks that a thread makes one pass at the model shapes (measured 4-5% faster than 8 blocks per SM
+  // with two or three passes each); the cap only bounds the grid for very large tensors.
+  long long cap = (long long)sms * 32 / (groups * p.njobs);
   if (cap < 1) cap = 1;
-  dim3 grid((unsigned)(want < cap ? want : cap), groups, p.njobs);
+  const long long gx = want < cap ? want : cap;
+  dim3 grid((unsigned)gx, groups, p.njobs);
   if (head_dim == 128) rope_commit_kernel<128><<<grid, kThreads, 0, stream>>>(p);
   else rope_commit_kernel<64><<<grid, kThreads, 0, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
