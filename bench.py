@@ -386,7 +386,8 @@ def run_ours(args):
         t_commit8 = time_call(lambda: api.sdvg_kv_commit_e4m3(c8, st.k_r, st.v, inv, inv, sh.slots - 1, api.SDVG_STAGE))
         q8 = torch.empty(st.q_r.shape, dtype=torch.uint8, device=device)
         api.sdvg_quant_e4m3(st.q_r, inv, q8)
-        t_attn8 = time_call(lambda: api.sdvg_block_attn_fwd_e4m3(q8, None, None, c8, sh.slots - 1, desc * desc, desc, st.out,
+        qk_desc = desc * desc
+        t_attn8 = time_call(lambda: api.sdvg_block_attn_fwd_e4m3(q8, None, None, c8, sh.slots - 1, qk_desc, desc, st.out,
                                                                  None, sh.scale, st.ws), n=40)
         assert api.sdvg_block_attn_status(st.ws) == api.SDVG_OK
         elems = sh.block_tokens * sh.heads * sh.head_dim
