@@ -353,6 +353,19 @@ int sdvg_kv_commit_e4m3(sdvg_cache* cache, const void* k_roped, const void* v, c
                         void* stream);
 
 /*
+ * sdvg_rope3d_qk_commit for an 8-bit ring, one pass: q8_out = e4m3(rope(q) * q_inv_scale), e4m3(rope(k) *
+ * k_inv_scale) and e4m3(v * v_inv_scale) go into the ring slot of block_index.  rope() is the bit-specified
+ * rotation of sdvg_rope3d_qk INCLUDING its rounding to bf16, so the result is bit-identical to
+ * sdvg_rope3d_qk followed by sdvg_quant_e4m3 (q) and sdvg_kv_commit_e4m3 (k, v).  q, k, v: device bf16
+ * [block_tokens, heads, 128]; q8_out: device bytes, same shape; q / q8_out / q_inv_scale may be NULL together.
+ * Other arguments and errors as sdvg_rope3d_qk_commit; BAD_SHAPE for a bf16 ring.
+ */
+int sdvg_rope3d_qk_commit_e4m3(sdvg_cache* cache, const void* q, const void* k, const void* v, void* q8_out,
+                               const float* q_inv_scale, const float* k_inv_scale, const float* v_inv_scale,
+                               int frames, int grid_h, int grid_w, int frame_offset, const float* cos_sin_tab,
+                               int tab_frames, int64_t block_index, int flags, int64_t* evicted_block, void* stream);
+
+/*
  * sdvg_block_attn_fwd on E4M3 operands:
  *   out[i, h, :] = v_descale[h] * sum_j softmax_j(scale * qk_descale[h] * <dec q[i,h,:], dec K[j,h,:]>) dec V[j,h,:]
  * with the same visible keys.  q8, k_self8, v_self8: device bytes [block_tokens, heads, 128] (k_self8 and

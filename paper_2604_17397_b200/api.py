@@ -64,6 +64,8 @@ SIGNATURES = {
     "sdvg_cache_bytes_e4m3": (_SZ, [_I, _I, _I, _I]),
     "sdvg_cache_create_e4m3": (_I, [C.POINTER(_VP), _VP, _VP, _I, _I, _I, _I]),
     "sdvg_kv_commit_e4m3": (_I, [_VP, _VP, _VP, _VP, _VP, _I64, _I, C.POINTER(_I64), _VP]),
+    "sdvg_rope3d_qk_commit_e4m3": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
+                                        C.POINTER(_I64), _VP]),
     "sdvg_block_attn_fwd_e4m3": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
 }
 
@@ -394,6 +396,21 @@ def sdvg_kv_commit_e4m3(cache: Cache, k_roped, v, k_inv_scale, v_inv_scale, bloc
                                    _scales(k_inv_scale, cache.heads), _scales(v_inv_scale, cache.heads), block_index,
                                    flags, C.byref(ev), _stream(stream))
     _check(st, "sdvg_kv_commit_e4m3")
+    return ev.value
+
+
+def sdvg_rope3d_qk_commit_e4m3(cache: Cache, q, k, v, q8_out, q_inv_scale, k_inv_scale, v_inv_scale, grid,
+                               frame_offset: int, table, tab_frames: int, block_index: int, flags: int, stream=None) -> int:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    frames, grid_h, grid_w = grid
+    ev = _I64(-1)
+    st = lib().sdvg_rope3d_qk_commit_e4m3(cache.handle, _bf16(q, None if q is None else shape), _bf16(k, shape),
+                                          _bf16(v, shape), _u8(q8_out, None if q8_out is None else shape),
+                                          None if q_inv_scale is None else _scales(q_inv_scale, cache.heads),
+                                          _scales(k_inv_scale, cache.heads), _scales(v_inv_scale, cache.heads),
+                                          frames, grid_h, grid_w, frame_offset, _ptr(table), tab_frames, block_index,
+                                          flags, C.byref(ev), _stream(stream))
+    _check(st, "sdvg_rope3d_qk_commit_e4m3")
     return ev.value
 
 

@@ -10,6 +10,7 @@
 #include <cuda_bf16.h>
 
 #include "sdvg_internal.h"
+#include "sm100_ptx.cuh"
 
 namespace {
 
@@ -22,6 +23,10 @@ struct TensorJob {
   uint4* dst_logical;      // same layout, or nullptr
   uint4* dst_slot;         // points at (head 0, slot, token 0): head stride = slots*tokens*dim, or nullptr
   int rope;                // rotate pairs (q, k) or copy (v)
+  // 8-bit variant: the (rotated, bf16-rounded) values times inv_scale[head] as E4M3 bytes, 8 per thread
+  uint2* q8_logical;       // [tokens, heads, dim] bytes, or nullptr
+  uint2* q8_slot;          // ring slot of a byte ring (same strides, counted in 8-byte units), or nullptr
+  const float* inv_scale;  // [heads]
 };
 
 struct RopeCommitParams {
@@ -48,7 +53,13 @@ __device__ __forceinline__ uint32_t rotate_pair(uint32_t w, float2 cs) {
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
-template <int D>
+// two bf16 pairs -> four E4M3 bytes, element order kept
+__device__ __forceinline__ uint32_t quant4(uint32_t w0, uint32_t w1, float inv) {
+  return sm100::pack_e4m3x4(__fmul_rn(bf16_lo(w0), inv), __fmul_rn(bf16_hi(w0), inv), __fmul_rn(bf16_lo(w1), inv),
+                            __fmul_rn(bf16_hi(w1), inv));
+}
+
+template <int D, bool Q8 = false>
 __global__ void __launch_bounds__(kThreads) rope_commit_kernel(const __grid_constant__ RopeCommitParams p) {
   constexpr int VPR = D / 8;                       // 16-byte vectors per (token, head) row
   const TensorJob job = p.job[blockIdx.z];
@@ -93,6 +104,12 @@ __global__ void __launch_bounds__(kThreads) rope_commit_kernel(const __grid_cons
         if (job.dst_logical) __stcs(job.dst_logical + row0 + (size_t)g * VPR, w);
         if (job.dst_slot)
           job.dst_slot[(size_t)(h0 + g) * p.slot_head_stride_vec + (size_t)t * VPR + j] = w;
+        if constexpr (Q8) {
+          const float inv = __ldg(job.inv_scale + h0 + g);
+          const uint2 o = make_uint2(quant4(w.x, w.y, inv), quant4(w.z, w.w, inv));
+          if (job.q8_logical) job.q8_logical[row0 + (size_t)g * VPR] = o;
+          if (job.q8_slot) job.q8_slot[(size_t)(h0 + g) * p.slot_head_stride_vec + (size_t)t * VPR + j] = o;
+        }
       }
     }
   }
@@ -140,7 +157,7 @@ int fill_rope(RopeCommitParams& p, int head_dim, int tokens, const RopeArgs& r) 
   return SDVG_OK;
 }
 
-int launch(RopeCommitParams& p, int head_dim, cudaStream_t stream) {
+int launch(RopeCommitParams& p, int head_dim, cudaStream_t stream, bool q8 = false) {
   if (p.njobs == 0) return SDVG_OK;
   const int vpr = head_dim / 8;
   const long long total = (long long)p.tokens * vpr;
@@ -156,7 +173,8 @@ int launch(RopeCommitParams& p, int head_dim, cudaStream_t stream) {
   if (cap < 1) cap = 1;
   const long long gx = want < cap ? want : cap;
   dim3 grid((unsigned)gx, groups, p.njobs);
-  if (head_dim == 128) rope_commit_kernel<128><<<grid, kThreads, 0, stream>>>(p);
+  if (q8) rope_commit_kernel<128, true><<<grid, kThreads, 0, stream>>>(p);      // a byte ring has head_dim 128
+  else if (head_dim == 128) rope_commit_kernel<128><<<grid, kThreads, 0, stream>>>(p);
   else rope_commit_kernel<64><<<grid, kThreads, 0, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
 }
@@ -233,6 +251,38 @@ int sdvg_rope3d_qk_commit(sdvg_cache* c, const void* q, const void* k, const voi
   p.job[p.njobs++] = TensorJob{(const uint4*)k, (uint4*)k_out, kslot, 1};
   p.job[p.njobs++] = TensorJob{(const uint4*)v, nullptr, vslot, 0};
   st = launch(p, c->head_dim, (cudaStream_t)stream);
+  if (st != SDVG_OK) return st;
+  sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
+  return SDVG_OK;
+}
+
+int sdvg_rope3d_qk_commit_e4m3(sdvg_cache* c, const void* q, const void* k, const void* v, void* q8_out,
+                               const float* q_inv_scale, const float* k_inv_scale, const float* v_inv_scale,
+                               int frames, int grid_h, int grid_w, int frame_offset, const float* cos_sin_tab,
+                               int tab_frames, int64_t block_index, int flags, int64_t* evicted_block, void* stream) {
+  if (!c || !k || !v || !k_inv_scale || !v_inv_scale) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 1) return SDVG_ERR_BAD_SHAPE;
+  if ((q == nullptr) != (q8_out == nullptr) || (q && !q_inv_scale)) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(q) || !sdvg::aligned16(k) || !sdvg::aligned16(v) || !sdvg::aligned16(q8_out) ||
+      ((reinterpret_cast<uintptr_t>(q_inv_scale) | reinterpret_cast<uintptr_t>(k_inv_scale) |
+        reinterpret_cast<uintptr_t>(v_inv_scale)) & 3))
+    return SDVG_ERR_MISALIGNED;
+  RopeCommitParams p = {};
+  p.tokens = c->block_tokens;
+  p.heads = c->heads;
+  int st = fill_rope(p, c->head_dim, c->block_tokens,
+                     RopeArgs{frames, grid_h, grid_w, frame_offset, tab_frames, cos_sin_tab});
+  if (st != SDVG_OK) return st;
+  int slot = 0;
+  if ((st = sdvg::ring_begin_commit(c, block_index, flags, &slot)) != SDVG_OK) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  p.slot_head_stride_vec = (long long)c->slots * c->block_tokens * (c->head_dim / 8);    // in 8-byte units here
+  uint2* kslot = (uint2*)c->k_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  uint2* vslot = (uint2*)c->v_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  if (q) p.job[p.njobs++] = TensorJob{(const uint4*)q, nullptr, nullptr, 1, (uint2*)q8_out, nullptr, q_inv_scale};
+  p.job[p.njobs++] = TensorJob{(const uint4*)k, nullptr, nullptr, 1, nullptr, kslot, k_inv_scale};
+  p.job[p.njobs++] = TensorJob{(const uint4*)v, nullptr, nullptr, 0, nullptr, vslot, v_inv_scale};
+  st = launch(p, c->head_dim, (cudaStream_t)stream, true);
   if (st != SDVG_OK) return st;
   sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
   return SDVG_OK;

@@ -37,19 +37,54 @@ class ModelState:
     tab_frames: int
     scale: float
     workspace: torch.Tensor = None
+    # 8-bit ring (cache.e4m3): static inverse scales per head, device fp32 [heads]
+    q_inv_scale: torch.Tensor = None
+    k_inv_scale: torch.Tensor = None
+    v_inv_scale: torch.Tensor = None
 
     def __post_init__(self):
         if self.workspace is None:
             self.workspace = api.attn_workspace(device=self.table.device)
         shape = (self.cache.block_tokens, self.cache.heads, self.cache.head_dim)
         dev = self.table.device
-        self.q_roped = torch.empty(shape, dtype=torch.bfloat16, device=dev)
-        self.k_roped = torch.empty(shape, dtype=torch.bfloat16, device=dev)
+        self.e4m3 = bool(getattr(self.cache, "e4m3", False))
+        if self.e4m3:
+            if self.q_inv_scale is None or self.k_inv_scale is None or self.v_inv_scale is None:
+                raise ValueError("an 8-bit ring needs q, k and v inverse scales")
+            self.qk_descale = 1.0 / (self.q_inv_scale * self.k_inv_scale)
+            self.v_descale = 1.0 / self.v_inv_scale
+        # the roped queries of the current step: bf16, or E4M3 codes for an 8-bit ring
+        self.q_roped = torch.empty(shape, dtype=torch.uint8 if self.e4m3 else torch.bfloat16, device=dev)
         self.out = torch.empty(shape, dtype=torch.bfloat16, device=dev)
 
     @property
     def frames(self) -> int:
         return self.grid[0]
+
+    def new_q_roped(self) -> torch.Tensor:
+        return torch.zeros_like(self.q_roped)
+
+    def stage_and_attend(self, q, k, v, block: int, q_roped, out) -> None:
+        """One denoise step of `block`: fused rope (+ quantise) + stage, then attention against the ring."""
+        if self.e4m3:
+            api.sdvg_rope3d_qk_commit_e4m3(self.cache, q, k, v, q_roped, self.q_inv_scale, self.k_inv_scale,
+                                           self.v_inv_scale, self.grid, block * self.frames, self.table,
+                                           self.tab_frames, block, api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd_e4m3(q_roped, None, None, self.cache, block, self.qk_descale, self.v_descale, out,
+                                         None, self.scale, self.workspace)
+        else:
+            api.sdvg_rope3d_qk_commit(self.cache, q, k, v, q_roped, None, self.grid, block * self.frames, self.table,
+                                      self.tab_frames, block, api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd(q_roped, None, None, self.cache, block, out, None, self.scale, self.workspace)
+
+    def commit_final(self, k, v, block: int) -> int:
+        """Rope the block's final K and write it with V into the ring (SDVG_FINAL); returns the evicted block."""
+        if self.e4m3:
+            return api.sdvg_rope3d_qk_commit_e4m3(self.cache, None, k, v, None, None, self.k_inv_scale, self.v_inv_scale,
+                                                  self.grid, block * self.frames, self.table, self.tab_frames, block,
+                                                  api.SDVG_FINAL)
+        return api.sdvg_rope3d_qk_commit(self.cache, None, k, v, None, None, self.grid, block * self.frames, self.table,
+                                         self.tab_frames, block, api.SDVG_FINAL)
 
 
 @dataclass
@@ -66,18 +101,14 @@ class TraceResult:
 def _denoise(model: str, m: ModelState, block: int, steps: int, provider, on_attention) -> int:
     for s in range(steps):
         q, k, v = provider(model, block, "step", s)
-        api.sdvg_rope3d_qk_commit(m.cache, q, k, v, m.q_roped, None, m.grid, block * m.frames, m.table,
-                                  m.tab_frames, block, api.SDVG_STAGE)
-        api.sdvg_block_attn_fwd(m.q_roped, None, None, m.cache, block, m.out, None, m.scale, m.workspace)
+        m.stage_and_attend(q, k, v, block, m.q_roped, m.out)
         if on_attention is not None:
             on_attention(model, block, s, m.q_roped, m.out)
     return steps
 
 
 def _commit_clean(m: ModelState, block: int, k, v) -> int:
-    """Rope the block's final K and write it with V into the ring (SDVG_FINAL)."""
-    return api.sdvg_rope3d_qk_commit(m.cache, None, k, v, None, None, m.grid, block * m.frames, m.table,
-                                     m.tab_frames, block, api.SDVG_FINAL)
+    return m.commit_final(k, v, block)
 
 
 def run_schedule(num_blocks: int, steps: int, scores: torch.Tensor, tau: float,
@@ -93,7 +124,9 @@ def run_schedule(num_blocks: int, steps: int, scores: torch.Tensor, tau: float,
               model's shape; kind is "step" (one denoise step), "clean" (the model's final
               K/V, q is None) or "accepted" (target-shaped K/V of an accepted draft block)
     on_attention  optional ``f(model, block, step, q_roped, out)`` called after each
-              attention launch (the tensors are reused by the next step)
+              attention launch (the tensors are reused by the next step; q_roped holds E4M3
+              codes when the model's ring is an 8-bit one)
+    A model whose ``cache`` is an 8-bit ring takes every step through the _e4m3 entry points.
     The accept decision is read back to the host once per block, which is the only
     synchronisation point of the flow.
     """
@@ -143,7 +176,7 @@ class BlockStepGraph:
         dev = m.table.device
         new = lambda: torch.zeros(shape, dtype=torch.bfloat16, device=dev)
         self.q, self.k, self.v = ([new() for _ in range(steps)] for _ in range(3))
-        self.q_roped = [new() for _ in range(steps)]
+        self.q_roped = [m.new_q_roped() for _ in range(steps)]
         self.out = [new() for _ in range(steps)]
         self.m, self.block, self.steps = m, block, steps
         self._run()                                   # warm-up, eager
@@ -155,9 +188,7 @@ class BlockStepGraph:
     def _run(self):
         m, b = self.m, self.block
         for s in range(self.steps):
-            api.sdvg_rope3d_qk_commit(m.cache, self.q[s], self.k[s], self.v[s], self.q_roped[s], None, m.grid,
-                                      b * m.frames, m.table, m.tab_frames, b, api.SDVG_STAGE)
-            api.sdvg_block_attn_fwd(self.q_roped[s], None, None, m.cache, b, self.out[s], None, m.scale, m.workspace)
+            m.stage_and_attend(self.q[s], self.k[s], self.v[s], b, self.q_roped[s], self.out[s])
 
     def replay(self):
         self.graph.replay()

@@ -129,6 +129,15 @@ def test_e4m3_entry_points_validate_on_the_host(lib):
     assert commit8(h8, 0x30000, 0x40000, None, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_INVALID_ARG
     assert commit8(h8, 0x30008, 0x40000, sc, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_MISALIGNED
     assert commit8(h8, 0x30000, 0x40000, sc + 2, sc, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_MISALIGNED
+    fused8 = lib.sdvg_rope3d_qk_commit_e4m3
+    tab = 0x80000
+    assert fused8(h16, None, 0x30000, 0x40000, None, None, sc, sc, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert fused8(h8, 0x50000, 0x30000, 0x40000, None, sc, sc, sc, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert fused8(h8, 0x50000, 0x30000, 0x40000, 0x60000, None, sc, sc, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert fused8(h8, None, 0x30000, 0x40000, None, None, sc, sc, 1, 8, 7, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert fused8(h8, None, 0x30000, 0x40000, None, None, sc, sc, 1, 8, 8, 4, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_STATE
+    assert fused8(h8, None, 0x30000, 0x40000, None, None, sc, sc, 1, 8, 8, 0, tab, 4, 2, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_STATE
+    assert fused8(h8, None, 0x30008, 0x40000, None, None, sc, sc, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_MISALIGNED
     ws = lib.sdvg_block_attn_workspace_bytes()
     f8, f16 = lib.sdvg_block_attn_fwd_e4m3, lib.sdvg_block_attn_fwd
     assert f8(0x50000, 0x30000, 0x40000, h16, 0, sc, sc, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_SHAPE

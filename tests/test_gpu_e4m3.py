@@ -241,3 +241,120 @@ def test_full_size_target_shape_sampled_rows():
         bound = p_rounding_bound(q8, k_all, v_all, sc * sc, sc, sh.scale, [h], rows)
         check_attention(out[rows, h], o_ref[:, 0], bound[:, 0], ("14b", h))
     cache.close()
+
+
+def test_fused_rope_quantise_stage_is_bit_identical_to_the_separate_calls_and_the_oracle():
+    sh = synth.Shape("e4m3-prologue", heads=5, head_dim=128, frames=2, grid_h=6, grid_w=11, slots=3)
+    grid = (sh.frames, sh.grid_h, sh.grid_w)
+    tabf = 4 * sh.frames
+    tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+    ref_tab = O.rope_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w)
+    fused = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True)
+    apart = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True)
+    rng = np.random.default_rng(4)
+    q_inv, k_inv, v_inv = (rng.uniform(20, 120, sh.heads).astype(np.float32) for _ in range(3))
+    for b in range(4):
+        q, k, v = (synth.block_tensor(sh, 21, b, 0, t, std=1.5) for t in (synth.Q, synth.K, synth.V))
+        dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
+        for flags in (api.SDVG_STAGE, api.SDVG_FINAL):
+            q8 = torch.zeros(q.shape, dtype=torch.uint8, device="cuda")
+            ev = api.sdvg_rope3d_qk_commit_e4m3(fused, dq, dk, dv, q8, f32_dev(q_inv), f32_dev(k_inv), f32_dev(v_inv), grid,
+                                                b * sh.frames, tab, tabf, b, flags)
+            # the same in three calls
+            q_r, k_r = torch.empty_like(dq), torch.empty_like(dk)
+            api.sdvg_rope3d_qk(dq, dk, q_r, k_r, grid, b * sh.frames, tab, tabf)
+            q8b = torch.zeros_like(q8)
+            api.sdvg_quant_e4m3(q_r, f32_dev(q_inv), q8b)
+            ev2 = api.sdvg_kv_commit_e4m3(apart, k_r, dv, f32_dev(k_inv), f32_dev(v_inv), b, flags)
+            assert ev == ev2 and fused.state() == apart.state()
+            assert torch.equal(q8, q8b)
+            fk, fv = fused.read_block(b % sh.slots)
+            ak, av = apart.read_block(b % sh.slots)
+            assert torch.equal(fk, ak) and torch.equal(fv, av)
+            # and the oracle: bit-specified rotation rounded to bf16, then the quantiser
+            qr = O.rope_bitspec(q, grid, b * sh.frames, ref_tab, tabf)
+            kr = O.rope_bitspec(k, grid, b * sh.frames, ref_tab, tabf)
+            assert np.array_equal(q8.cpu().numpy(), O.quant_e4m3_ref(qr, q_inv))
+            assert np.array_equal(fk.cpu().numpy(), O.quant_e4m3_ref(kr, k_inv))
+            assert np.array_equal(fv.cpu().numpy(), O.quant_e4m3_ref(v, v_inv))
+    # k and v alone (no q), and a bf16 ring is refused
+    api.sdvg_rope3d_qk_commit_e4m3(fused, None, dk, dv, None, None, f32_dev(k_inv), f32_dev(v_inv), grid, 0, tab, tabf, 4,
+                                   api.SDVG_STAGE)
+    bf = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    with pytest.raises(api.SdvgError) as e:
+        api.sdvg_rope3d_qk_commit_e4m3(bf, None, dk, dv, None, None, f32_dev(k_inv), f32_dev(v_inv), grid, 0, tab, tabf, 0,
+                                       api.SDVG_STAGE)
+    assert e.value.status == api.SDVG_ERR_BAD_SHAPE
+
+
+def test_schedule_with_8bit_rings_follows_the_flow_and_holds_the_oracle_codes():
+    from paper_2604_17397_b200 import schedule
+    from test_gpu_schedule import Provider
+
+    sh_d = synth.Shape("d8", heads=3, head_dim=128, frames=3, grid_h=4, grid_w=13, slots=3)
+    sh_t = synth.Shape("t8", heads=5, head_dim=128, frames=3, grid_h=4, grid_w=13, slots=4)
+    B, steps, tau, seed = 9, 2, -0.7, 61
+    tabf = B * sh_t.frames
+    scores = synth.calibrated_scores(B, 12, seed)
+    prov = Provider(sh_d, sh_t, seed)
+    rng = np.random.default_rng(seed)
+    models, inv = {}, {}
+    for name, sh in (("drafter", sh_d), ("target", sh_t)):
+        inv[name] = [rng.uniform(60, 110, sh.heads).astype(np.float32) for _ in range(3)]
+        cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True)
+        tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+        models[name] = schedule.ModelState(cache, (sh.frames, sh.grid_h, sh.grid_w), tab, tabf, sh.scale,
+                                           q_inv_scale=f32_dev(inv[name][0]), k_inv_scale=f32_dev(inv[name][1]),
+                                           v_inv_scale=f32_dev(inv[name][2]))
+    shapes = {"drafter": sh_d, "target": sh_t}
+    checked = []
+
+    def on_attention(model, b, s, q8, out):
+        if (b + s) % 3:
+            return
+        m, sh = models[model], shapes[model]
+        # the window as the device ring holds it at this moment, the staged block included
+        ks, vs = [], []
+        for blk in range(max(0, b - (sh.slots - 1)), b + 1):
+            gk, gv = m.cache.read_block(blk % sh.slots)
+            ks.append(gk.cpu().numpy())
+            vs.append(gv.cpu().numpy())
+        k_all, v_all = np.concatenate(ks), np.concatenate(vs)
+        r = np.random.default_rng([seed, b, s])
+        heads = list(np.sort(r.choice(sh.heads, 2, replace=False)))
+        rows = np.sort(r.choice(sh.block_tokens, 16, replace=False))
+        qkd = 1.0 / (inv[model][0].astype(np.float64) * inv[model][1])
+        vd = 1.0 / inv[model][2].astype(np.float64)
+        q8n = q8.cpu().numpy()
+        o_ref, _ = O.attn_e4m3_ref(q8n, k_all, v_all, qkd, vd, sh.scale, heads=heads, rows=rows)
+        bound = p_rounding_bound(q8n, k_all, v_all, qkd, vd, sh.scale, heads, rows)
+        got = out[torch.from_numpy(rows).cuda()][:, torch.tensor(heads).cuda()]
+        check_attention(got, o_ref, bound, (model, b, s))
+        checked.append((model, b, s))
+
+    res = schedule.run_schedule(B, steps, torch.from_numpy(scores).cuda(), tau, models["drafter"], models["target"],
+                                prov.device, on_attention=on_attention)
+    for m in models.values():
+        assert api.sdvg_block_attn_status(m.workspace) == api.SDVG_OK
+    assert len(checked) >= 6 and {c[0] for c in checked} == {"drafter", "target"}
+
+    # the flow (routing, branches, evictions, call counts) is that of the oracle's schedule; its bf16 rings,
+    # quantised with the same scales, are what the 8-bit rings must hold
+    rd = O.RingCacheRef(sh_d.slots, sh_d.heads, sh_d.block_tokens, sh_d.head_dim)
+    rt = O.RingCacheRef(sh_t.slots, sh_t.heads, sh_t.block_tokens, sh_t.head_dim)
+    want = O.schedule_ref(B, steps, scores, tau, rd, rt, prov.bits, (sh_d.frames, sh_d.grid_h, sh_d.grid_w),
+                          (sh_t.frames, sh_t.grid_h, sh_t.grid_w), sh_t.frames,
+                          O.rope_table(128, tabf, sh_d.grid_h, sh_d.grid_w), O.rope_table(128, tabf, sh_t.grid_h, sh_t.grid_w),
+                          tabf)
+    assert np.array_equal(res.accept, want.accept) and res.target_source == want.target_source
+    assert 0 < int(want.accept.sum()) < B - 1
+    assert res.drafter_evicted == want.drafter_evicted and res.target_evicted == want.target_evicted
+    assert res.drafter_attn_calls == want.drafter_attn_calls and res.target_attn_calls == want.target_attn_calls
+    for name, ref in (("drafter", rd), ("target", rt)):
+        cache = models[name].cache
+        assert cache.state()[:2] == (ref.next_block, ref.slot_block)
+        for s in range(ref.slots):
+            gk, gv = cache.read_block(s)
+            assert np.array_equal(gk.cpu().numpy(), O.quant_e4m3_ref(ref.k[s], inv[name][1])), (name, s)
+            assert np.array_equal(gv.cpu().numpy(), O.quant_e4m3_ref(ref.v[s], inv[name][2])), (name, s)
+        cache.close()
