@@ -358,3 +358,36 @@ def test_schedule_with_8bit_rings_follows_the_flow_and_holds_the_oracle_codes():
             assert np.array_equal(gk.cpu().numpy(), O.quant_e4m3_ref(ref.k[s], inv[name][1])), (name, s)
             assert np.array_equal(gv.cpu().numpy(), O.quant_e4m3_ref(ref.v[s], inv[name][2])), (name, s)
         cache.close()
+
+
+def test_block_steps_of_an_8bit_ring_replayed_from_a_cuda_graph_equal_the_eager_calls():
+    from paper_2604_17397_b200 import schedule
+
+    sh = synth.Shape("graph8", heads=3, head_dim=128, frames=3, grid_h=6, grid_w=11, slots=3)
+    tabf, steps = 4 * sh.frames, 3
+    inv = [f32_dev(np.full(sh.heads, x, dtype=np.float32)) for x in (90.0, 100.0, 80.0)]
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True)
+    tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+    m = schedule.ModelState(cache, (sh.frames, sh.grid_h, sh.grid_w), tab, tabf, sh.scale,
+                            q_inv_scale=inv[0], k_inv_scale=inv[1], v_inv_scale=inv[2])
+    for b in range(3):                                  # block 2 sees two committed blocks
+        if b == 2:
+            g = schedule.BlockStepGraph(m, b, steps)
+            eager, eager_q8 = [], []
+            for s in range(steps):
+                q, k, v = (to_dev(synth.block_tensor(sh, 98, b, s, t)) for t in (synth.Q, synth.K, synth.V))
+                g.q[s].copy_(q); g.k[s].copy_(k); g.v[s].copy_(v)
+                m.stage_and_attend(q, k, v, b, m.q_roped, m.out)
+                eager.append(m.out.clone())
+                eager_q8.append(m.q_roped.clone())
+            for o in g.out:
+                o.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            assert api.sdvg_block_attn_status(m.workspace) == api.SDVG_OK
+            for s in range(steps):
+                assert torch.equal(g.q_roped[s], eager_q8[s]), s
+                assert torch.equal(g.out[s].view(torch.int16), eager[s].view(torch.int16)), s
+        k, v = (to_dev(synth.block_tensor(sh, 98, b, 9, t)) for t in (synth.K, synth.V))
+        m.commit_final(k, v, b)
+    cache.close()
