@@ -155,9 +155,20 @@ int sdvg_rope3d_qk_commit(sdvg_cache* cache, const void* q, const void* k, const
 /*
  * Device scratch needed by sdvg_block_attn_fwd (a few hundred bytes: a work
  * counter and a status word).  256-byte aligned, caller-owned, must not be
- * shared by calls that overlap on the device.
+ * shared by calls that overlap on the device.  The status word is STICKY: a
+ * kernel whose bounded wait gave up raises it to SDVG_ERR_TIMEOUT and no later
+ * launch lowers it again, so one check after a sequence of steps (before their
+ * results are committed) is enough.  Clear a new workspace, and a workspace whose
+ * error has been handled, with sdvg_block_attn_workspace_reset.
  */
 size_t sdvg_block_attn_workspace_bytes(void);
+
+/*
+ * Zeroes the workspace on `stream` (a memset, no kernel).  Call it once after
+ * allocating the buffer and again after a reported SDVG_ERR_TIMEOUT has been dealt with.
+ * Errors: INVALID_ARG (NULL or too small), MISALIGNED, CUDA.
+ */
+int sdvg_block_attn_workspace_reset(void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * out[i, h, :] = sum_j softmax_j(scale * <q[i,h,:], K[j,h,:]>) V[j,h,:] where j
@@ -199,11 +210,21 @@ int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* con
                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Synchronises `stream` and reports what the last attention launch that used
- * `workspace` left in its status word: SDVG_OK, or SDVG_ERR_TIMEOUT if a
- * bounded wait inside the kernel gave up (the output is then undefined).
+ * Synchronises `stream` and reports the status word of `workspace`: SDVG_OK, or
+ * SDVG_ERR_TIMEOUT if a bounded wait inside ANY attention launch on this
+ * workspace since its last reset gave up (the outputs of that launch and of
+ * everything computed from them are then undefined).  Reading does not clear it.
  */
 int sdvg_block_attn_status(const void* workspace, void* stream);
+
+/*
+ * Diagnostic: synchronises `stream` and writes to *events (host) how many times, since the last reset of
+ * `workspace`, a warp of an attention kernel took the path that rescales the output accumulator because the
+ * reference maximum of one of its query rows moved (the online-softmax correction; with the lazy reference
+ * it is rare on ordinary data and frequent when the logits keep rising along the keys).  Tests use it to
+ * prove that this path ran.
+ */
+int sdvg_block_attn_rescale_events(const void* workspace, unsigned long long* events, void* stream);
 
 /*
  * Self-test of the bounded device-side wait (no counterpart in the paper; it backs the promise that a
@@ -233,11 +254,15 @@ int sdvg_selftest_bounded_wait(void* workspace, size_t workspace_bytes, unsigned
  *   - First call on a device: the function looks up where that device's copy of the array
  *     lives (cudaGetSymbolAddress, with the device current) and remembers it.  Make that first
  *     call outside of any stream capture.
- *   - All calls on a device share the one array.  Each call clears it on `stream` before the
- *     kernel runs and the kernel leaves its status word there, so two calls that overlap on
- *     the GPU (different streams, no ordering between them) race on it; keep them ordered.
+ *   - All calls on a device share the one array and it keeps what the last call left in it.
+ *     It starts out zeroed (static initialisation), nothing in it has to be zero at the start
+ *     of a call, and the only thing a kernel leaves there is the sticky status word, so no
+ *     call clears it.  Two calls that overlap on the GPU (different streams, no ordering
+ *     between them) share that word: a timeout is then reported without telling which of
+ *     them it was; keep them ordered if that matters.
  *   - *scratch_device_ptr (optional, host) receives the device address of the array, which
- *     can be given to sdvg_block_attn_status to read the status word after the call.
+ *     can be given to sdvg_block_attn_status to read the status word after the call and to
+ *     sdvg_block_attn_workspace_reset (256 bytes) to clear a handled error.
  * Arguments, results and errors are otherwise those of sdvg_block_attn_fwd.
  */
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self,
@@ -259,6 +284,11 @@ int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v
  * With frame_offsets == NULL frames_per_block must be >= 1; with offsets every
  * block must own at least one frame (checked on the device: a block with none
  * gets accept 0, q_min NaN, argmin -1).
+ * The offsets must be non-decreasing and the scores buffer must hold at least
+ * offsets[num_blocks] floats.  The host cannot read them, so the kernel trusts only
+ * the two ends: it never reads outside [offsets[0], offsets[num_blocks]), and a block
+ * whose own range runs backwards or leaves that interval is treated as a block
+ * without frames.
  * Errors: INVALID_ARG, BAD_SHAPE (num_blocks < 0, frames_per_block < 1).
  */
 int sdvg_route(const float* scores, const int32_t* frame_offsets,

@@ -51,10 +51,12 @@ SIGNATURES = {
     "sdvg_rope3d_qk_commit": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
                                    C.POINTER(_I64), _VP]),
     "sdvg_block_attn_workspace_bytes": (_SZ, []),
+    "sdvg_block_attn_workspace_reset": (_I, [_VP, _SZ, _VP]),
     "sdvg_block_attn_fwd": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_attn_fwd_batched": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_selftest_bounded_wait": (_I, [_VP, _SZ, C.c_ulonglong, _VP]),
     "sdvg_block_attn_status": (_I, [_VP, _VP]),
+    "sdvg_block_attn_rescale_events": (_I, [_VP, C.POINTER(C.c_ulonglong), _VP]),
     "sdvg_block_attn_fwd_noalloc": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _F, C.POINTER(_VP), _VP]),
     "sdvg_route": (_I, [_VP, _VP, _I, _I, _I64, _F, _VP, _VP, _VP, _VP]),
     "sdvg_route_policy": (_I, [_VP, _VP, _I, _I, _I64, _I, _F, _I, _I, _I, _VP, _F, _VP, _VP, _VP, _VP]),
@@ -234,10 +236,24 @@ def sdvg_rope3d_qk_commit(cache: Cache, q, k, v, q_out, k_out, grid, frame_offse
 # ---------------------------------------------------------------- attention
 
 def attn_workspace(device="cuda", extra_bytes: int = 0) -> torch.Tensor:
+    """A 256-byte-aligned attention workspace on `device`, cleared through the library."""
     n = lib().sdvg_block_attn_workspace_bytes() + extra_bytes
-    raw = torch.zeros(n + 256, dtype=torch.uint8, device=device)
+    raw = torch.empty(n + 256, dtype=torch.uint8, device=device)
     off = (-raw.data_ptr()) % 256
-    return raw[off:off + n]
+    ws = raw[off:off + n]
+    with torch.cuda.device(ws.device):
+        sdvg_block_attn_workspace_reset(ws)
+    return ws
+
+
+def sdvg_block_attn_workspace_reset(workspace, nbytes: Optional[int] = None, stream=None) -> None:
+    """Clears the workspace (and with it a sticky SDVG_ERR_TIMEOUT).  `workspace` is a tensor, or an
+    integer device address together with `nbytes`."""
+    if isinstance(workspace, int):
+        ptr, n = workspace, int(nbytes)
+    else:
+        ptr, n = workspace.data_ptr(), workspace.numel()
+    _check(lib().sdvg_block_attn_workspace_reset(ptr, n, _stream(stream)), "sdvg_block_attn_workspace_reset")
 
 
 def sdvg_block_attn_fwd(q, k_self, v_self, cache: Cache, block_index: int, out, lse, scale: float,
@@ -287,6 +303,14 @@ def sdvg_block_attn_status(workspace, stream=None) -> int:
     returned by sdvg_block_attn_fwd_noalloc."""
     ptr = workspace if isinstance(workspace, int) else workspace.data_ptr()
     return lib().sdvg_block_attn_status(ptr, _stream(stream))
+
+
+def sdvg_block_attn_rescale_events(workspace, stream=None) -> int:
+    """Warp-level accumulator-rescale events recorded in the workspace since its last reset."""
+    ptr = workspace if isinstance(workspace, int) else workspace.data_ptr()
+    n = C.c_ulonglong(0)
+    _check(lib().sdvg_block_attn_rescale_events(ptr, C.byref(n), _stream(stream)), "sdvg_block_attn_rescale_events")
+    return int(n.value)
 
 
 def sdvg_block_attn_fwd_noalloc(q, k_self, v_self, cache: Cache, block_index: int, out, lse, scale: float,

@@ -20,7 +20,6 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
-#include <stdlib.h>
 
 #include <mutex>
 
@@ -57,12 +56,9 @@ struct alignas(64) AttnParams {
   int nseg;
   int tokens, heads;
   float scale_log2e;                   // scale * log2(e): softmax is evaluated with exp2
-  unsigned int* work;                  // [0] work counter, [1] status word
+  unsigned int* work;                  // [0] self-test result, [1] sticky status word, [2] count of accumulator rescale events
   const float* qk_descale;             // 8-bit variant only: per head, q scale * k scale
   const float* v_descale;              // 8-bit variant only: per head, v scale
-#ifdef SDVG_ATTN_DEBUG
-  float* dbg;                          // S, P, O of the first key tile of CTA (0, 0)
-#endif
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -84,7 +80,8 @@ struct Deadline {
 };
 
 // Slow path of the bounded wait: poll until the phase completes or the deadline passes.  Kept out
-// of line of the first attempt so that the timer read never sits on the fast path.
+// of line of the first attempt so that the timer read never sits on the fast path.  (A suspend-time
+// hint on the try_wait makes the waiting threads poll less often but wake later: measured slower.)
 __device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity, uint64_t deadline_ns,
                                            unsigned int* status) {
   uint32_t ok;
@@ -104,7 +101,7 @@ __device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity
       : "=r"(ok)
       : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
       : "memory");
-  if (!ok) atomicExch(status, (unsigned)SDVG_ERR_TIMEOUT);
+  if (!ok) atomicMax(status, (unsigned)SDVG_ERR_TIMEOUT);      // sticky: only a reset clears it
   return ok != 0;
 }
 
@@ -121,214 +118,6 @@ __device__ __forceinline__ bool wait_warp(uint64_t* bar, uint32_t parity, const 
   return __all_sync(0xffffffffu, wait_bar(bar, parity, d));
 }
 
-template <int D>
-struct SimpleSmem {
-  static constexpr int kHalves = D / 64;                 // 64-column (128-byte) swizzle panels
-  static constexpr int kPanelBytes = kTileN * 128;       // 128 rows x 128 B
-  static constexpr int kTileBytes = kHalves * kPanelBytes;
-  static constexpr int kQ = 0;
-  static constexpr int kK = kTileBytes;
-  static constexpr int kV = 2 * kTileBytes;
-  static constexpr int kBars = 3 * kTileBytes;
-  static constexpr int kTotal = kBars + 64;
-  static constexpr int kDynamic = kTotal + 1024;         // slack for the 1024-byte alignment
-};
-
-// One CTA = one 128-row query tile of one head, four warps, no overlap between the stages.
-template <int D>
-__global__ void __launch_bounds__(128, 1) attn_fwd_simple_kernel(const __grid_constant__ AttnParams p) {
-  using L = SimpleSmem<D>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + L::kBars);
-  uint64_t* s_bar = full_bar + 1;
-  uint64_t* o_bar = full_bar + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(full_bar + 3);
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int qt = blockIdx.x, head = blockIdx.y;
-  const AttnProblem& pr = p.prob[blockIdx.z];
-  constexpr uint32_t kTmemCols = 256;                    // S: [0,128) (P aliases its first 64), O: [128, 128+D)
-
-  if (tid == 0) {
-    mbar_init(full_bar, 1);
-    mbar_init(s_bar, 1);
-    mbar_init(o_bar, 1);
-    fence_mbar_init();
-    prefetch_tmap(&pr.q_map);
-  }
-  if (warp == 0) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base, tO = tmem_base + 128;
-  const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-  const Deadline wc{globaltimer_ns() + kWaitLimitNs, p.work + 1};
-
-  uint32_t full_phase = 0, s_phase = 0, o_phase = 0;
-  bool alive = true;
-
-  if (tid == 0) {
-    mbar_expect_tx(full_bar, L::kTileBytes);
-    for (int h = 0; h < L::kHalves; ++h)
-      tma_load_3d(smem + L::kQ + h * L::kPanelBytes, &pr.q_map, full_bar, h * 64, qt * kTileM, head);
-  }
-  alive = wait_bar(full_bar, full_phase, wc);
-  full_phase ^= 1;
-
-  constexpr uint32_t kIdescQK = idesc_bf16_f32(kTileM, kTileN, false);
-  constexpr uint32_t kIdescPV = idesc_bf16_f32(kTileM, D, true);
-  const uint32_t sQ = smem_u32(smem + L::kQ), sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
-
-  float m_run = -INFINITY, l_run = 0.f;
-  int it = 0;
-  for (int seg = 0; seg < p.nseg && alive; ++seg) {
-    const int len = p.seg_len[seg];
-    const int ntiles = (len + kTileN - 1) / kTileN;
-    for (int kt = 0; kt < ntiles && alive; ++kt, ++it) {
-      const int valid = min(kTileN, len - kt * kTileN);
-      if (tid == 0) {
-        mbar_expect_tx(full_bar, 2 * L::kTileBytes);
-        for (int h = 0; h < L::kHalves; ++h) {
-          tma_load_3d(smem + L::kK + h * L::kPanelBytes, &pr.k_map[seg], full_bar, h * 64, kt * kTileN, head);
-          tma_load_3d(smem + L::kV + h * L::kPanelBytes, &pr.v_map[seg], full_bar, h * 64, kt * kTileN, head);
-        }
-      }
-      if (!(alive = wait_bar(full_bar, full_phase, wc))) break;
-      full_phase ^= 1;
-      if (tid == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * L::kPanelBytes + (kk & 3) * 32;   // 16 bf16 = 32 B along K
-          mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), kIdescQK,
-                 kk > 0);
-        }
-        mma_commit(s_bar);
-      }
-      if (!(alive = wait_bar(s_bar, s_phase, wc))) break;
-      s_phase ^= 1;
-      tc_fence_after();
-
-      // ---- softmax of this thread's row ---------------------------------------------------
-      uint32_t s[4][32];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, s[c]);
-      tmem_wait_ld();
-#ifdef SDVG_ATTN_DEBUG
-      if (p.dbg && qt == 0 && head == 0 && it == 0)
-        for (int c = 0; c < 4; ++c)
-          for (int j = 0; j < 32; ++j) p.dbg[tid * 128 + c * 32 + j] = __uint_as_float(s[c][j]);
-#endif
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float x = __uint_as_float(s[c][j]) * p.scale_log2e;
-          if (c * 32 + j >= valid) x = -INFINITY;
-          s[c][j] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
-        }
-      const float m_new = fmaxf(m_run, mx);
-      const float alpha = fast_exp2(m_run - m_new);
-      float sum = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float p0 = fast_exp2(__uint_as_float(s[c][2 * j]) - m_new);
-          const float p1 = fast_exp2(__uint_as_float(s[c][2 * j + 1]) - m_new);
-          sum += p0 + p1;
-          __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-          pk[j] = *reinterpret_cast<uint32_t*>(&b);
-        }
-        tmem_st16(tS + lane_off + c * 16, pk);     // P overwrites S columns already held in registers
-      }
-      l_run = l_run * alpha + sum;
-      m_run = m_new;
-      if (it > 0) {
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tO + lane_off + c * 32, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-          tmem_st32(tO + lane_off + c * 32, o);
-        }
-      }
-      tmem_wait_st();
-      tc_fence_before();
-      __syncthreads();
-      if (tid == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < kTileN / 16; ++kk) {
-          // 16 keys = two 8-row groups of the V panel; the two 64-column panels are kPanelBytes apart
-          mma_ts(tO, tS + kk * 8, smem_desc_sw128(sV + kk * 2048, L::kPanelBytes, 1024), kIdescPV,
-                 (it > 0 || kk > 0) ? 1u : 0u);
-        }
-        mma_commit(o_bar);
-      }
-      if (!(alive = wait_bar(o_bar, o_phase, wc))) break;
-      o_phase ^= 1;
-      tc_fence_after();
-#ifdef SDVG_ATTN_DEBUG
-      if (p.dbg && qt == 0 && head == 0 && it == 0) {
-        for (int c = 0; c < 2; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tS + lane_off + c * 32, r);
-          tmem_wait_ld();
-          for (int j = 0; j < 32; ++j) p.dbg[128 * 128 + tid * 64 + c * 32 + j] = __uint_as_float(r[j]);
-        }
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(tO + lane_off + c * 32, r);
-          tmem_wait_ld();
-          for (int j = 0; j < 32; ++j) p.dbg[128 * 128 + 128 * 64 + tid * D + c * 32 + j] = __uint_as_float(r[j]);
-        }
-      }
-#endif
-    }
-  }
-
-  // ---- epilogue: O / l -> bf16, this thread's row ------------------------------------------
-  const int row = qt * kTileM + tid;
-  if (alive && it > 0) {
-    const float inv = 1.f / l_run;
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t o[32];
-      tmem_ld32(tO + lane_off + c * 32, o);
-      tmem_wait_ld();
-      if (row < p.tokens) {
-        uint4* dst = reinterpret_cast<uint4*>(pr.out + ((size_t)row * p.heads + head) * D + c * 32);
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(o[v * 8 + 2 * e]) * inv,
-                                                     __uint_as_float(o[v * 8 + 2 * e + 1]) * inv);
-            w[e] = *reinterpret_cast<uint32_t*>(&b);
-          }
-          dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-    }
-    if (pr.lse && row < p.tokens)
-      pr.lse[(size_t)head * p.tokens + row] = m_run * 0.6931471805599453f + logf(l_run);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
-}
-
 #include "attn_fwd_ws.cuh"
 
 // ---- host side -------------------------------------------------------------------------------
@@ -338,14 +127,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
+  // looked up once; the initialisation of a function-local static is thread-safe
+  static const EncodeTiledFn fn = [] {
     void* ptr = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
+      return reinterpret_cast<EncodeTiledFn>(ptr);
+    return (EncodeTiledFn) nullptr;
+  }();
   return fn;
 }
 
@@ -365,32 +155,31 @@ int make_map(CUtensorMap* m, const void* base, int head_dim, long long rows, int
   return r == CUDA_SUCCESS ? SDVG_OK : SDVG_ERR_CUDA;
 }
 
-template <int D>
-int launch_simple(const AttnParams& p, cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_simple_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SimpleSmem<D>::kDynamic);
-    if (e != cudaSuccess) return sdvg::cuda_status(e);
-    configured = true;
-  }
-  dim3 grid((p.tokens + kTileM - 1) / kTileM, p.heads, p.batch);
-  attn_fwd_simple_kernel<D><<<grid, 128, SimpleSmem<D>::kDynamic, stream>>>(p);
-  return sdvg::cuda_status(cudaGetLastError());
-}
+// One-time set-up per device and kernel instance: the opt-in to the kernel's dynamic shared memory is a
+// per-device attribute, and the grid is sized by that device's SM count.
+constexpr int kMaxDevices = 64;
+std::mutex g_setup_mu;
 
 template <int D, bool F8 = false>
 int launch_ws(const AttnParams& p, cudaStream_t stream) {
-  static bool configured = false;
-  static int sms = 0;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         WsCfg<D, F8>::kDynamic);
-    if (e != cudaSuccess) return sdvg::cuda_status(e);
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    configured = true;
+  static int sms_of_device[kMaxDevices] = {};          // 0: this device has not been set up yet
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  if (dev < 0 || dev >= kMaxDevices) return SDVG_ERR_INVALID_ARG;
+  int sms;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (!sms_of_device[dev]) {
+      e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               WsCfg<D, F8>::kDynamic);
+      if (e != cudaSuccess) return sdvg::cuda_status(e);
+      int n = 0;
+      e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+      if (e != cudaSuccess || n < 1) return sdvg::cuda_status(e != cudaSuccess ? e : cudaErrorUnknown);
+      sms_of_device[dev] = n;
+    }
+    sms = sms_of_device[dev];
   }
   const int total_tiles = ((p.tokens + kTileM - 1) / kTileM) * p.heads * p.batch;
   const int grid = total_tiles < sms ? total_tiles : sms;
@@ -398,16 +187,6 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
   return sdvg::cuda_status(cudaGetLastError());
 }
 
-bool use_simple_kernel() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("SDVG_ATTN_KERNEL");
-    v = (e && e[0] == 's') ? 1 : 0;
-  }
-  return v == 1;
-}
-
-// Validation, tensor maps, scratch clear and launch shared by the attention entry points.
 // Argument and ring-state checks of one problem; touches no CUDA API.
 int check_problem(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c, int64_t block_index,
                   const void* out, const float* lse) {
@@ -510,16 +289,8 @@ int attn_forward_batch(int batch, const void* const* q, const void* const* k_sel
     same = same && nseg[b] == nseg[0];
     for (int s = 0; same && s < nseg[b]; ++s) same = seg_len[b][s] == seg_len[0][s];
   }
-#ifdef SDVG_ATTN_DEBUG
-  p.dbg = workspace_bytes >= (size_t)kWorkspaceBytes + 4 * (128 * 128 + 128 * 64 + 128 * 128)
-              ? (float*)((char*)workspace + kWorkspaceBytes)
-              : nullptr;
-#endif
-  cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceBytes, stream);
-  if (e != cudaSuccess) return sdvg::cuda_status(e);
   auto launch = [&](const AttnParams& pp) {
     if (elem_bytes == 1) return launch_ws<128, true>(pp, stream);     // an 8-bit cache always has head_dim 128
-    if (use_simple_kernel()) return D == 128 ? launch_simple<128>(pp, stream) : launch_simple<64>(pp, stream);
     return D == 128 ? launch_ws<128>(pp, stream) : launch_ws<64>(pp, stream);
   };
   if (same) {
@@ -577,6 +348,12 @@ int sdvg_debug_set_trace(void* p) { return (int)cudaMemcpyToSymbol(g_trace, &p, 
 
 size_t sdvg_block_attn_workspace_bytes(void) { return kWorkspaceBytes; }
 
+int sdvg_block_attn_workspace_reset(void* workspace, size_t workspace_bytes, void* stream_) {
+  if (!workspace || workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return SDVG_ERR_MISALIGNED;
+  return sdvg::cuda_status(cudaMemsetAsync(workspace, 0, kWorkspaceBytes, (cudaStream_t)stream_));
+}
+
 int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
                         int64_t block_index, void* out, float* lse, float scale, void* workspace,
                         size_t workspace_bytes, void* stream_) {
@@ -609,7 +386,6 @@ int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
                                 int64_t block_index, void* out, float* lse, float scale,
                                 void** scratch_device_ptr, void* stream_) {
-  constexpr int kMaxDevices = 64;
   static std::mutex mu;
   static void* scratch_of_device[kMaxDevices] = {};
   // The built-in scratch has a fixed size; refuse rather than overrun if the kernel ever needs more.
@@ -656,6 +432,17 @@ int sdvg_block_attn_status(const void* workspace, void* stream_) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) return sdvg::cuda_status(e);
   return w[1] == 0 ? SDVG_OK : (int)w[1];
+}
+
+int sdvg_block_attn_rescale_events(const void* workspace, unsigned long long* events, void* stream_) {
+  if (!workspace || !events) return SDVG_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  unsigned int w[3] = {0, 0, 0};
+  cudaError_t e = cudaMemcpyAsync(w, workspace, sizeof(w), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return sdvg::cuda_status(e);
+  *events = w[2];
+  return SDVG_OK;
 }
 
 }  // extern "C"

@@ -73,19 +73,27 @@ struct WsCfg {
   static constexpr int kHalves = F8 ? D / 128 : D / 64;             // 128-byte panels per row
   static constexpr int kPanelBytes = 128 * 128;
   static constexpr int kTileBytes = kHalves * kPanelBytes;          // one Q, K or V tile
-  static constexpr int kStages = (D == 128 && !F8) ? 5 : 8;         // K/V ring entries (K and V alternate)
+  static constexpr int kStages = (D == 128 && !F8) ? 4 : 8;         // K/V ring entries (K and V alternate)
   static constexpr int kPanelElems = F8 ? 128 : 64;                 // elements per panel row
   static constexpr int kQ = 0;                                      // two query tiles
   static constexpr int kKV = 2 * kTileBytes;
-  static constexpr int kRowState = kKV + kStages * kTileBytes;      // float [2][128]: -m*c2 of a row, later the helper's l
-  static constexpr int kMerge = kRowState + 2 * 128 * 4;            // float [128]: lane 1's -m*c2 when a split tile is merged
-  static constexpr int kBars = kMerge + 128 * 4;
+  static constexpr int kRowMax = kKV + kStages * kTileBytes;        // float [2 parities][2 lanes][2 halves][128]: partial row maxima
+  static constexpr int kRowSum = kRowMax + 2 * 2 * 2 * 128 * 4;     // float [2 lanes][128]: the upper half's share of the row sum
+  static constexpr int kMerge = kRowSum + 2 * 128 * 4;              // float [2][128]: lane 1's -m*c2 and l when a split tile is merged
+  static constexpr int kBars = kMerge + 2 * 128 * 4;
   static constexpr int kNumBars = 20 + 2 * kStages;
   static constexpr int kMisc = kBars + kNumBars * 8;                // tmem slot
   static constexpr int kTotal = kMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;
-  static constexpr int kThreads = 512;
+  static constexpr int kSoftmaxWarps = 16;                          // 2 lanes x 2 column halves x 4 warps
+  static constexpr int kThreads = (kSoftmaxWarps + 4) * 32;         // + TMA producer, the two MMA issuers, one idle warp
   static constexpr uint32_t kTmemCols = 512;
+  // Registers.  Warp w runs on SM sub-partition w % 4, each of which has 16384 registers: four softmax warps and
+  // one of warps 16-19 share one.  The CTA is launched with kLaunchRegs per thread; the softmax warps then grow
+  // to kSoftmaxRegs out of what the fifth warp gives back (setmaxnreg).
+  static constexpr int kLaunchRegs = 96, kSoftmaxRegs = 112, kIssueRegs = 32;
+  static_assert(5 * 32 * kLaunchRegs <= 16384, "register file of a sub-partition");
+  static_assert(4 * kSoftmaxRegs + kIssueRegs <= 5 * kLaunchRegs, "register pool of a sub-partition");
   static_assert(kDynamic <= 232448, "shared memory budget");
 };
 
@@ -213,23 +221,43 @@ __device__ __forceinline__ void exp2_poly2(uint64_t x2, float& e0, float& e1) {
   e1 = __uint_as_float(__float_as_uint(t1) * 0x00800000u + __float_as_uint(p1));
 }
 
-// Out of every 4 consecutive element pairs of a row, this many take the polynomial path.
-#ifndef SDVG_ATTN_POLY_PAIRS
-#define SDVG_ATTN_POLY_PAIRS 0
+// Share of the exponentials that goes to the FMA pipe, per role: out of every 4 consecutive element pairs
+// of a 32-column chunk this many take the polynomial (4 = the whole chunk).
+#ifndef SDVG_MIX_HELPER
+#define SDVG_MIX_HELPER 0
 #endif
-
-#ifndef SDVG_ATTN_POLY_PAIRS_F8
-#define SDVG_ATTN_POLY_PAIRS_F8 0
+#ifndef SDVG_MIX_SOFTMAX
+#define SDVG_MIX_SOFTMAX 0
 #endif
+#ifndef SDVG_MIX_SOFTMAX_MID
+#define SDVG_MIX_SOFTMAX_MID 0
+#endif
+#ifndef SDVG_MIX_HELPER_F8
+#define SDVG_MIX_HELPER_F8 0
+#endif
+#ifndef SDVG_MIX_SOFTMAX_F8
+#define SDVG_MIX_SOFTMAX_F8 0
+#endif
+#ifndef SDVG_MIX_SOFTMAX_MID_F8
+#define SDVG_MIX_SOFTMAX_MID_F8 0
+#endif
+template <bool F8>
+struct ExpMix {
+  static constexpr int kHelper = F8 ? SDVG_MIX_HELPER_F8 : SDVG_MIX_HELPER;            // key columns 96-127
+  static constexpr int kSoftmax = F8 ? SDVG_MIX_SOFTMAX_F8 : SDVG_MIX_SOFTMAX;         // key columns 0-63
+  static constexpr int kSoftmaxMid = F8 ? SDVG_MIX_SOFTMAX_MID_F8 : SDVG_MIX_SOFTMAX_MID;   // key columns 64-95
+};
 
 // One 32-column chunk of a row: P = 2^(c2 * S - m*c2) as bf16 pairs, returns the packed partial row sums.
+// POLY of every 4 consecutive element pairs take the polynomial path (4: the whole chunk).
+template <int POLY>
 __device__ __forceinline__ void exp_chunk(const uint32_t (&s)[32], uint64_t c2x2, uint64_t negx2, uint32_t (&pk)[16],
                                           uint64_t& sum_a, uint64_t& sum_b) {
 #pragma unroll
   for (int k = 0; k < 16; ++k) {
     const uint64_t x2 = fma2(pack2(__uint_as_float(s[2 * k]), __uint_as_float(s[2 * k + 1])), c2x2, negx2);
     float p0, p1;
-    if ((k & 3) < SDVG_ATTN_POLY_PAIRS) {
+    if ((k & 3) < POLY) {
       exp2_poly2(x2, p0, p1);
     } else {
       float x0, x1;
@@ -245,6 +273,7 @@ __device__ __forceinline__ void exp_chunk(const uint32_t (&s)[32], uint64_t c2x2
 }
 
 // The same chunk as E4M3 bytes (four per word); the row sums are taken before the rounding, as above.
+template <int POLY>
 __device__ __forceinline__ void exp_chunk_f8(const uint32_t (&s)[32], uint64_t c2x2, uint64_t negx2, uint32_t (&pk)[8],
                                              uint64_t& sum_a, uint64_t& sum_b) {
 #pragma unroll
@@ -254,7 +283,7 @@ __device__ __forceinline__ void exp_chunk_f8(const uint32_t (&s)[32], uint64_t c
     for (int u = 0; u < 2; ++u) {
       const uint64_t x2 =
           fma2(pack2(__uint_as_float(s[4 * k + 2 * u]), __uint_as_float(s[4 * k + 2 * u + 1])), c2x2, negx2);
-      if (((2 * k + u) & 3) < SDVG_ATTN_POLY_PAIRS_F8) {
+      if (((2 * k + u) & 3) < POLY) {
         exp2_poly2(x2, e[2 * u], e[2 * u + 1]);
       } else {
         float x0, x1;
@@ -287,27 +316,40 @@ __device__ __forceinline__ void max_chunk(const uint32_t (&s)[32], float (&mx)[4
       mx[u] = fmax3(mx[u], __uint_as_float(s[k + 2 * u]), __uint_as_float(s[k + 2 * u + 1]));
 }
 
+// Number of real keys in key tile `kt` of the concatenated key segments (the last tile of a segment may be ragged).
+__device__ __forceinline__ int key_tile_valid(const AttnParams& p, int kt) {
+  int valid = kTileN;
+  for (int seg = 0; seg < p.nseg; ++seg) {
+    const int nt = (p.seg_len[seg] + kTileN - 1) / kTileN;
+    if (kt < nt) {
+      valid = min(kTileN, p.seg_len[seg] - kt * kTileN);
+      break;
+    }
+    kt -= nt;
+  }
+  return valid;
+}
+
 template <int D, bool F8 = false>
-__global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_constant__ AttnParams p) {
+__global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(const __grid_constant__ AttnParams p) {
   using C = WsCfg<D, F8>;
+  using Mix = ExpMix<F8>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  // [2][128]: while an item runs, -m_ref * c2 of the row (softmax -> helper); at its end the helper's
-  // share of the row sum travels back through the same word
-  float* s_neg = reinterpret_cast<float*>(smem + C::kRowState);
-  float* s_lhelp = s_neg;
+  float* s_rowmax = reinterpret_cast<float*>(smem + C::kRowMax);
+  float* s_rowsum = reinterpret_cast<float*>(smem + C::kRowSum);
   float* s_merge = reinterpret_cast<float*>(smem + C::kMerge);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBars);
   uint64_t* q_full = bars;            // [2] TMA -> MMA
   uint64_t* q_empty = bars + 2;       // [2] MMA -> TMA
-  uint64_t* s_full = bars + 4;        // [2] MMA -> softmax
-  uint64_t* p_lo = bars + 6;          // [2] P columns 0-63 (softmax), 96-127 + O rescaled (helper) -> MMA, 256 arrivals
-  uint64_t* p_mid = bars + 8;         // [2] P columns 64-95 stored (softmax) -> MMA, 128 arrivals
-  uint64_t* row_ready = bars + 12;    // [2] softmax -> helper: -m*c2 of the row published, 128 arrivals
-  uint64_t* o_full = bars + 14;       // [2] MMA -> helper / softmax epilogue
-  uint64_t* l_ready = bars + 16;      // [2] helper -> softmax epilogue: its share of the row sum, 128 arrivals
-  uint64_t* lane1_done = bars + 18;   // softmax of lane 1 -> softmax of lane 0: partial result of a split tile published, 128 arrivals
-  uint64_t* merge_done = bars + 19;   // softmax of lane 0 -> softmax of lane 1: O_1 has been read, 128 arrivals
+  uint64_t* s_full = bars + 4;        // [2] MMA -> softmax: S holds lane i's logits
+  uint64_t* p_ready = bars + 6;       // [2] softmax -> MMA: P_i stored (and O_i rescaled), 256 arrivals
+  uint64_t* mx_ready = bars + 8;      // [2] softmax <-> softmax: both partial row maxima published, 256 arrivals
+  uint64_t* s_free = bars + 10;       // softmax -> MMA: the row of S is in registers, 256 arrivals
+  uint64_t* sum_ready = bars + 12;    // [2] upper half -> lower half: its share of the row sum, 128 arrivals
+  uint64_t* o_full = bars + 14;       // [2] MMA -> softmax: O_i += P_i V has completed
+  uint64_t* lane1_done = bars + 18;   // lane 1 -> lane 0: partial result of a split tile published, 128 arrivals
+  uint64_t* merge_done = bars + 19;   // lane 0 -> lane 1: O_1 has been read, 128 arrivals
   uint64_t* kv_full = bars + 20;      // [kStages]
   uint64_t* kv_empty = kv_full + C::kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kMisc);
@@ -319,12 +361,12 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       mbar_init(&q_full[i], 1);
       mbar_init(&q_empty[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_lo[i], 256);
-      mbar_init(&p_mid[i], 128);
-      mbar_init(&row_ready[i], 128);
+      mbar_init(&p_ready[i], 256);
+      mbar_init(&mx_ready[i], 256);
+      mbar_init(&sum_ready[i], 128);
       mbar_init(&o_full[i], 1);
-      mbar_init(&l_ready[i], 128);
     }
+    mbar_init(s_free, 256);
     mbar_init(lane1_done, 128);
     mbar_init(merge_done, 128);
     for (int s = 0; s < C::kStages; ++s) {
@@ -348,6 +390,8 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // tensor memory columns: O_0, O_1 (128 each), S (128, shared by the two lanes), P_0, P_1 (64 each)
+  constexpr uint32_t kColO = 0, kColS = 256, kColP = 384;
   // Every wait of this kernel gives up at the same absolute time; a thread that gives up records
   // the timeout and leaves its role loop, and all roles meet at the common exit below.
   const Deadline dl{globaltimer_ns() + kWaitLimitNs, p.work + 1};
@@ -355,10 +399,10 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
   int ntiles_k = 0;
   for (int s = 0; s < p.nseg; ++s) ntiles_k += (p.seg_len[s] + kTileN - 1) / kTileN;
 
-  if (warp >= 12) {
+  if (warp >= C::kSoftmaxWarps) {
     // ================= producer / issuer warps: few registers ==================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
-    if (warp == 12) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kIssueRegs));
+    if (warp == C::kSoftmaxWarps) {
       // ---- TMA producer -------------------------------------------------------------------
       const bool leader = elect_one();
       uint32_t q_cnt[2] = {0, 0}, kv_issued = 0;
@@ -404,16 +448,16 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
                           &q_full[i], h * C::kPanelElems, it.tile[i] * kTileM, it.head[i] % p.heads);
           }
         }
-        // K/V tiles in the order the issuer consumes them: K of the first key tile of every stream, then
-        // step by step and lane by lane V of this step and K of the next
+        // K/V tiles in the order the issuers consume them: K of the first key tile of every stream, then
+        // step by step and lane by lane K of the next step and V of this one
         const int streams = it.dual ? it.lanes : 1;
         for (int s = 0; s < streams && alive; ++s) load_kv(false, it.head[s], it.key_tile(s, 0));
         #pragma unroll 1
         for (int t = 0; t < it.nk[0] && alive; ++t)
           for (int s = 0; s < streams && alive; ++s) {
             if (t >= it.nk[s]) continue;
-            load_kv(true, it.head[s], it.key_tile(s, t));
-            if (t + 1 < it.nk[s] && alive) load_kv(false, it.head[s], it.key_tile(s, t + 1));
+            if (t + 1 < it.nk[s]) load_kv(false, it.head[s], it.key_tile(s, t + 1));
+            if (alive) load_kv(true, it.head[s], it.key_tile(s, t));
           }
       }
       // Drain: every load issued above lands in this CTA's shared memory; do not exit under them.
@@ -422,67 +466,54 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         if (q_cnt[i] > 0) wait_warp(&q_full[i], (q_cnt[i] - 1) & 1, dl);
       for (uint32_t n = kv_issued > (uint32_t)C::kStages ? kv_issued - C::kStages : 0; n < kv_issued; ++n)
         wait_warp(&kv_full[n % C::kStages], (n / C::kStages) & 1, dl);
-    } else if (warp == 13) {
-      // ---- MMA issuer ---------------------------------------------------------------------
+    } else if (warp == C::kSoftmaxWarps + 1) {
+      // ---- MMA issuer, first product: S = Q_i K^T ------------------------------------------------
+      // The two products have an issuing warp each: while one warp sits in its waits and bookkeeping the
+      // other one's MMAs keep the tensor pipe fed (the pipe takes only a few instructions ahead).
       const bool leader = elect_one();
       constexpr uint32_t kIdescQK = F8 ? idesc_e4m3_f32(kTileM, kTileN, false) : idesc_bf16_f32(kTileM, kTileN, false);
-      constexpr uint32_t kIdescPV = F8 ? idesc_e4m3_f32(kTileM, D, true) : idesc_bf16_f32(kTileM, D, true);
       const uint32_t sQ = smem_u32(smem + C::kQ), sKV = smem_u32(smem + C::kKV);
       uint32_t q_cnt[2] = {0, 0};
-      uint32_t pv_par = 0;                 // bit i: phase parity of lane i's P barriers
-      RingPos ring;                        // next K/V stage to consume
+      uint32_t qk_cnt = 0;                 // products written into S so far = phase index of s_free
+      RingPos ring;                        // walks every entry of the K/V ring; this warp consumes the K tiles
       bool alive = true;
       SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
-
-      // Every instruction this warp executes between "P is ready" and the MMAs lengthens the chain that
-      // paces the kernel, so the issue loops are unrolled (descriptor offsets become immediates) while the
-      // loop over the two lanes stays rolled to keep the code this warp has to fetch small.
-      // S_i = Q_i K^T into TMEM columns [128 i, 128 i + 128)
       // Descriptors of stage 0 and of the two query tiles, built once; a stage or a 16-wide slice is then one
       // addition to the address field (all of this CTA's shared memory fits that field, so nothing carries out).
       const uint64_t descQ0 = smem_desc_sw128(sQ, 16, 1024);
       const uint64_t descK0 = smem_desc_sw128(sKV, 16, 1024);
-      const uint64_t descV0 = smem_desc_sw128(sKV, C::kPanelBytes, 1024);
-      auto issue_qk = [&](int i, uint32_t st) {
-        const uint32_t d = tmem_base + i * 128;
-        const uint64_t a = descQ0 + (uint64_t)(i * (C::kTileBytes >> 4));
-        const uint64_t b = descK0 + (uint64_t)(st * (C::kTileBytes >> 4));
-        uint32_t acc = 0;
+      // S_i(t) = Q_i K^T of the lane's t-th key tile, from the ring's next stage if the lane has one of its own
+      // (else from `st`, the stage the other lane just used); the previous occupant of S must have been read
+      // into registers by its softmax threads
+      auto qk_step = [&](int i, bool own, uint32_t& st, bool release_stage, bool last_of_item) {
+        if (own) {
+          st = ring.stage;
+          if (!(alive = wait_warp(&kv_full[st], ring.phase, dl))) return;
+          ring.template advance<C::kStages>();
+        }
+        if (qk_cnt > 0 && !(alive = wait_warp(s_free, (qk_cnt - 1) & 1, dl))) return;
+        ++qk_cnt;
+        SDVG_TRACE(2, 50000 + i * 1000);
+        tc_fence_after();
+        if (leader) {
+          const uint32_t d = tmem_base + kColS;
+          const uint64_t a = descQ0 + (uint64_t)(i * (C::kTileBytes >> 4));
+          const uint64_t b = descK0 + (uint64_t)(st * (C::kTileBytes >> 4));
+          uint32_t acc = 0;
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          if (F8 && kk >= D / 32) break;                   // an 8-bit MMA covers 32 dims
-          // one MMA reads 32 B of every row = 2 descriptor units within a 128-byte panel, panels kPanelBytes apart
-          const uint64_t off = (uint64_t)((kk >> 2) * (C::kPanelBytes >> 4) + (kk & 3) * 2);
-          if constexpr (F8) mma_ss_f8(d, a + off, b + off, kIdescQK, acc);
-          else mma_ss(d, a + off, b + off, kIdescQK, acc);
-          acc = 1;
+          for (int kk = 0; kk < D / 16; ++kk) {
+            if (F8 && kk >= D / 32) break;                   // an 8-bit MMA covers 32 dims
+            // one MMA reads 32 B of every row = 2 descriptor units within a 128-byte panel, panels kPanelBytes apart
+            const uint64_t off = (uint64_t)((kk >> 2) * (C::kPanelBytes >> 4) + (kk & 3) * 2);
+            if constexpr (F8) mma_ss_f8(d, a + off, b + off, kIdescQK, acc);
+            else mma_ss(d, a + off, b + off, kIdescQK, acc);
+            acc = 1;
+          }
+          mma_commit(&s_full[i]);
+          if (release_stage) mma_commit(&kv_empty[st]);
+          if (last_of_item) mma_commit(&q_empty[i]);
         }
-      };
-      // O_i (+)= P_i[:, 16 kk .. 16 kk + 16) V[16 kk .. 16 kk + 16, :] for kk in [k0, k1); P_i is read from
-      // the first 64 columns of S_i
-      auto issue_pv = [&](int i, uint32_t st, int k0, int k1, uint32_t acc) {
-        const uint32_t d = tmem_base + 256 + i * 128, a = tmem_base + i * 128;
-        const uint64_t b = descV0 + (uint64_t)(st * (C::kTileBytes >> 4));
-#pragma unroll
-        for (int kk = k0; kk < k1; ++kk) {
-          // slice kk of P is 8 TMEM columns (16 bf16 or 32 bytes per row); its keys are 16 or 32 rows of V
-          if constexpr (F8) mma_ts_f8(d, a + kk * 8, b + (uint64_t)(kk * (4096 >> 4)), kIdescPV, acc);
-          else mma_ts(d, a + kk * 8, b + (uint64_t)(kk * (2048 >> 4)), kIdescPV, acc);
-          acc = 1;
-        }
-      };
-      // slices of P per 32-column chunk of S: chunk c of the softmax is slices [c kPc, c kPc + kPc)
-      constexpr int kPc = F8 ? 1 : 2;
-      // Are the next `n` (1 or 2) stages of the ring filled?  Does not block (test_wait, not try_wait,
-      // which may suspend the thread for microseconds when the answer is no).
-      auto stages_filled = [&](int n) {
-        RingPos r = ring;
-        bool ok = mbar_test_wait(&kv_full[r.stage], r.phase);
-        if (n > 1) {
-          r.template advance<C::kStages>();
-          ok = mbar_test_wait(&kv_full[r.stage], r.phase) && ok;
-        }
-        return __all_sync(0xffffffffu, ok);
+        SDVG_TRACE(2, 60000 + i * 1000);
       };
 
       #pragma unroll 1
@@ -499,208 +530,105 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
           ++q_cnt[i];
         }
         if (!alive) break;
-        // ---- prologue: S_i(0) ------------------------------------------------------------------
         uint32_t stK = 0;
+        // ---- prologue: S_i(0) ------------------------------------------------------------------
 #pragma unroll 1
-        for (int i = 0; i < nl && alive; ++i) {
-          const bool own = (i == 0) || dual;                 // this lane takes a stage of its own
-          const bool last_user = dual || (i == nl - 1);
-          if (own) {
-            stK = ring.stage;
-            if (!(alive = wait_warp(&kv_full[stK], ring.phase, dl))) break;
-            ring.template advance<C::kStages>();
-            tc_fence_after();
-          }
-          if (leader) {
-            issue_qk(i, stK);
-            mma_commit(&s_full[i]);
-            if (last_user) mma_commit(&kv_empty[stK]);
-          }
-        }
-        // ---- main loop: step t of lane i works on that lane's t-th key tile --------------------------
-        // The stages of a step (V of this key tile, K of the next) are taken from the ring one step ahead, in
-        // the shadow of MMAs already queued: what is left at the start of a step is a look at `nx.filled`.
-        struct {
-          uint32_t stV, phV, stK, phK;
-          bool filled;
-        } nx = {0, 0, 0, 0, false};
-        auto take = [&](bool with_k) {
-          nx.stV = ring.stage;
-          nx.phV = ring.phase;
-          nx.filled = stages_filled(with_k ? 2 : 1);
-          ring.template advance<C::kStages>();
-          if (with_k) {
-            nx.stK = ring.stage;
-            nx.phK = ring.phase;
-            ring.template advance<C::kStages>();
-          }
-        };
-        take(nk0 > 1);                                       // for step (0, lane 0)
+        for (int i = 0; i < nl && alive; ++i)
+          qk_step(i, (i == 0) || dual, stK, dual || (i == nl - 1), (i == 0 ? nk0 : nk1) == 1);
+        // ---- step t of lane i: S_i(t+1), one key tile ahead of that lane's softmax -----------------
         #pragma unroll 1
         for (int t = 0; t < nk0 && alive; ++t) {
-          uint32_t stV = 0;
-          SDVG_TRACE(2, 100 + t);
-          // everything that depends on t alone is worked out here: each instruction inside the lane loop
-          // sits between "P is ready" and the next MMA
           const int nl_t = t < nk1 ? nl : 1;                 // a split tile with an odd number of key tiles ends on lane 0
-          const bool more0 = t + 1 < nk0, more1 = t + 1 < nk1;
 #pragma unroll 1
           for (int i = 0; i < nl_t && alive; ++i) {
-            const bool more = i == 0 ? more0 : more1;
+            const int nk_i = i == 0 ? nk0 : nk1;
+            const bool own = (i == 0) || dual;               // this lane has stages of its own
+            if (t + 1 < nk_i) qk_step(i, own, stK, dual || (i == nl - 1), t + 2 == nk_i);
+            if (own) ring.template advance<C::kStages>();    // V of this step: the other issuing warp's tile
+          }
+        }
+      }
+    } else if (warp == C::kSoftmaxWarps + 2) {
+      // ---- MMA issuer, second product: O_i += P_i V ----------------------------------------------
+      const bool leader = elect_one();
+      constexpr uint32_t kIdescPV = F8 ? idesc_e4m3_f32(kTileM, D, true) : idesc_bf16_f32(kTileM, D, true);
+      const uint32_t sKV = smem_u32(smem + C::kKV);
+      uint32_t pv_par = 0;                 // bit i: phase parity of lane i's P barrier
+      RingPos ring;                        // walks every entry of the K/V ring; this warp consumes the V tiles
+      bool alive = true;
+      SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
+      const uint64_t descV0 = smem_desc_sw128(sKV, C::kPanelBytes, 1024);
+      constexpr int kSlices = F8 ? 4 : 8;  // MMAs per key tile: 32 or 16 keys each
+
+      #pragma unroll 1
+      for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
+        WsItem it;
+        sched.get(v, ntiles_k, it);
+        const int nl = it.lanes;
+        const bool dual = it.dual;
+        const int nk0 = it.nk[0], nk1 = it.nk[1];
+        ring.template skip<C::kStages>(dual ? nl : 1);       // the K tiles of the prologue
+        uint32_t stV = 0;
+        #pragma unroll 1
+        for (int t = 0; t < nk0 && alive; ++t) {
+          const int nl_t = t < nk1 ? nl : 1;
+#pragma unroll 1
+          for (int i = 0; i < nl_t && alive; ++i) {
+            const int nk_i = i == 0 ? nk0 : nk1;
             const bool last_user = dual || (i == nl - 1);
-            if (i == 0 || dual) {                            // this lane has stages of its own
-              stV = nx.stV;
-              stK = nx.stK;
-              if (!nx.filled) {
-                if (!(alive = wait_warp(&kv_full[stV], nx.phV, dl))) break;
-                if (more && !(alive = wait_warp(&kv_full[stK], nx.phK, dl))) break;
-              }
+            if ((i == 0) || dual) {                          // this lane has stages of its own
+              if (t + 1 < nk_i) ring.template advance<C::kStages>();   // K of the next step
+              stV = ring.stage;
+              if (!(alive = wait_warp(&kv_full[stV], ring.phase, dl))) break;
+              ring.template advance<C::kStages>();
             }
-            SDVG_TRACE(2, 1000 + i * 1000 + t);
             const uint32_t par = (pv_par >> i) & 1;
             pv_par ^= 1u << i;
-            // P_i columns 0-63 and 96-127 stored, O_i rescaled (for t = 0: O_i was read out by the
+            // P_i stored and O_i rescaled where a row maximum moved (for t = 0: O_i was read out by the
             // epilogue of the previous item before its softmax threads arrived here)
-            if (!(alive = wait_warp(&p_lo[i], par, dl))) break;
-            SDVG_TRACE(2, 3000 + i * 1000 + t);
+            if (!(alive = wait_warp(&p_ready[i], par, dl))) break;
+            SDVG_TRACE(5, 3000 + i * 1000 + t);
             tc_fence_after();
             if (leader) {
-              issue_pv(i, stV, 3 * kPc, 4 * kPc, t > 0 ? 1u : 0u);
-              issue_pv(i, stV, 0, 2 * kPc, 1u);
-            }
-            // six MMAs are queued: take the stages of the next step that has stages of its own
-            {
-              const bool next_in_this_t = dual && (i + 1 < nl_t);
-              if (next_in_this_t) take(more1);
-              else if (more0 && (dual || i == nl_t - 1)) take(t + 2 < nk0);
-            }
-            if (!(alive = wait_warp(&p_mid[i], par, dl))) break;
-            SDVG_TRACE(2, 5000 + i * 1000 + t);
-            tc_fence_after();
-            if (leader) {
-              issue_pv(i, stV, 2 * kPc, 3 * kPc, 1u);
+              // O_i (+)= P_i[:, slice kk] V[slice kk, :]; slice kk of P is 8 TMEM columns (16 bf16 or 32 bytes per
+              // row), its keys are 16 or 32 rows of V
+              const uint32_t d = tmem_base + kColO + i * 128, a = tmem_base + kColP + i * 64;
+              const uint64_t b = descV0 + (uint64_t)(stV * (C::kTileBytes >> 4));
+              uint32_t acc = t > 0 ? 1u : 0u;
+#pragma unroll
+              for (int kk = 0; kk < kSlices; ++kk) {
+                if constexpr (F8) mma_ts_f8(d, a + kk * 8, b + (uint64_t)(kk * (4096 >> 4)), kIdescPV, acc);
+                else mma_ts(d, a + kk * 8, b + (uint64_t)(kk * (2048 >> 4)), kIdescPV, acc);
+                acc = 1;
+              }
               mma_commit(&o_full[i]);
               if (last_user) mma_commit(&kv_empty[stV]);
-              if (more) {
-                issue_qk(i, stK);
-                mma_commit(&s_full[i]);
-                if (last_user) mma_commit(&kv_empty[stK]);
-              } else {
-                mma_commit(&q_empty[i]);
-              }
             }
-            SDVG_TRACE(2, 9000 + i * 1000 + t);
+            SDVG_TRACE(5, 9000 + i * 1000 + t);
           }
         }
-      }
-    }
-  } else if (warp >= 8) {
-    // ================= helper warps =============================================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 96;");
-    const int row = tid - 256;
-    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS[2] = {tmem_base + lane_off, tmem_base + 128 + lane_off};
-    const uint32_t tO[2] = {tmem_base + 256 + lane_off, tmem_base + 384 + lane_off};
-    const float c2 = p.scale_log2e;
-    const uint64_t c2x2 = pack2(c2, c2);
-    uint64_t c2h[2] = {c2x2, c2x2};      // 8-bit variant: the logit scale carries the head's q and k scales
-    uint32_t cnt[2] = {0, 0};            // (item, key tile) steps done per lane = phase index of its barriers
-    bool alive = true;
-    SDVG_TRACE_DECL(blockIdx.x == 0 && tid == 256)
-    #pragma unroll 1
-    for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
-      WsItem it;
-      sched.get(v, ntiles_k, it);
-      float l_part[2] = {0.f, 0.f}, neg_prev[2] = {0.f, 0.f};
-      if constexpr (F8) {
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const float c = c2 * __ldg(p.qk_descale + it.head[i]);
-          c2h[i] = pack2(c, c);
-        }
-      }
-      #pragma unroll 1
-      for (int j = 0; j < it.nk[0] && alive; ++j) {          // step j of lane i: that lane's j-th key tile
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          if (i >= it.lanes || !alive) break;
-          if (j >= it.nk[i]) continue;
-          const uint32_t par = cnt[i] & 1;
-          if (!(alive = wait_bar(&row_ready[i], par, dl))) break;
-          const float neg = s_neg[i * 128 + row];
-          // the row's reference maximum moved iff -m*c2 changed; both sides derive the factor the same way
-          const bool moved = (j > 0) && (neg != neg_prev[i]);
-          const float alpha = moved ? fast_exp2(__fsub_rn(neg, neg_prev[i])) : 1.f;
-          neg_prev[i] = neg;
-          SDVG_TRACE(3, 1000 * i + j);
-          if (__any_sync(0xffffffffu, moved)) {
-            // PV_i(j-1) is commit number cnt[i] - 1 on o_full[i]
-            if (!(alive = wait_bar(&o_full[i], (cnt[i] - 1) & 1, dl))) break;
-            tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {          // rare path: keep its code small
-              uint32_t o[32];
-              tmem_ld32(tO[i] + c * 32, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-              tmem_st32(tO[i] + c * 32, o);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            l_part[i] *= alpha;
-          }
-          SDVG_TRACE(3, 20000 + 1000 * i + j);
-          // ---- this row's share of P: key columns 96-127 -------------------------------------
-          tc_fence_after();
-          uint32_t s3[32];
-          tmem_ld32(tS[i] + 96, s3);
-          tmem_wait_ld();
-          uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-          if constexpr (F8) {
-            uint32_t pk[8];
-            exp_chunk_f8(s3, c2h[i], pack2(neg, neg), pk, sum_a, sum_b);
-            tmem_st8(tS[i] + 24, pk);
-          } else {
-            uint32_t pk[16];
-            exp_chunk(s3, c2x2, pack2(neg, neg), pk, sum_a, sum_b);
-            tmem_st16(tS[i] + 48, pk);
-          }
-          {
-            float a0, a1, b0, b1;
-            unpack2(sum_a, a0, a1);
-            unpack2(sum_b, b0, b1);
-            l_part[i] += (a0 + a1) + (b0 + b1);
-          }
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&p_lo[i]);
-          SDVG_TRACE(3, 30000 + 1000 * i + j);
-          ++cnt[i];
-        }
-      }
-      if (!alive) break;
-      // hand the partial row sums to the softmax threads that normalise and store the rows
-#pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        if (i >= it.lanes) break;
-        s_lhelp[i * 128 + row] = l_part[i];
-        mbar_arrive(&l_ready[i]);
       }
     }
   } else {
     // ================= softmax warps ===========================================================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 176;");
-    const int i = warp >> 2;                       // lane (query tile) of this warpgroup
+    // Two threads per query row: warps 0-7 take key columns 0-63 of their lane's rows (warps 0-3 lane 0,
+    // warps 4-7 lane 1), warps 8-15 columns 64-127.  A warp reaches the 32 TMEM lanes of its position in its
+    // warpgroup, so the two threads of a row sit in warps w and w + 8.
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kSoftmaxRegs));
+    const int i = (warp >> 2) & 1;                 // lane (query tile)
+    const int half = warp >> 3;                    // 0: key columns 0-63 of every tile, 1: columns 64-127
     const int row = tid & 127;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem_base + i * 128 + lane_off;
-    const uint32_t tO = tmem_base + 256 + i * 128 + lane_off;
+    const uint32_t tS = tmem_base + kColS + lane_off + half * 64;
+    const uint32_t tP = tmem_base + kColP + i * 64 + lane_off + half * (F8 ? 16 : 32);
+    const uint32_t tO = tmem_base + kColO + i * 128 + lane_off;
+    float* const my_max = s_rowmax + (i * 2 + half) * 128 + row;           // + parity * 512
+    float* const other_max = s_rowmax + (i * 2 + (half ^ 1)) * 128 + row;
     float c2 = p.scale_log2e;
     uint64_t c2x2 = pack2(c2, c2);
     uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0, split_cnt = 0;
     bool alive = true;
-    SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0)
+    SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0 && (half == 0 || i == 0))
     #pragma unroll 1
     for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
       WsItem it;
@@ -715,110 +643,135 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
         c2x2 = pack2(c2, c2);
       }
       float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2 (+ the window shift)
-      {
-        #pragma unroll 1
-        for (int j = 0; j < my_nk && alive; ++j) {        // this lane's j-th key tile
-          // number of real keys in that tile: the last tile of a key segment may be ragged
-          int valid = kTileN;
-          {
-            int kt = it.key_tile(i, j);
-            for (int seg = 0; seg < p.nseg; ++seg) {
-              const int nt = (p.seg_len[seg] + kTileN - 1) / kTileN;
-              if (kt < nt) {
-                valid = min(kTileN, p.seg_len[seg] - kt * kTileN);
-                break;
-              }
-              kt -= nt;
-            }
-          }
-          SDVG_TRACE(i, 0 + j);
-          if (!(alive = wait_bar(&s_full[i], s_cnt & 1, dl))) break;
-          SDVG_TRACE(i, 1000 + j);
-          ++s_cnt;
-          tc_fence_after();
-          if (valid < kTileN) {
-            // Ragged last tile of a key segment (TMA zero-filled the missing keys): overwrite their
-            // columns of S with -inf in tensor memory, for this thread and for the helper thread of the
-            // row, which reads its columns after row_ready.  Rare, so a plain column-by-column loop.
-#pragma unroll 1
-            for (int c = valid; c < kTileN; ++c) tmem_st1(tS + c, 0xff800000u);
-            tmem_wait_st();
-          }
-          // ---- row maximum over all 128 columns; the second half streams in while the first is reduced
-          uint32_t s[3][32];
-          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          {
-            uint32_t s3[32];
-            tmem_ld32(tS + 96, s3);
-            tmem_ld32(tS, s[0]);
-            tmem_wait_ld();
-            tmem_ld32(tS + 32, s[1]);
-            tmem_ld32(tS + 64, s[2]);
-            max_chunk(s3, mx);
-            max_chunk(s[0], mx);
-          }
-          tmem_wait_ld();
-          SDVG_TRACE(i, 2000 + j);
-          max_chunk(s[1], mx);
-          max_chunk(s[2], mx);
-          const float mxa = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-          if (j == 0) {
-            m_ref = mxa;
-            neg = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
-          } else if ((mxa - m_ref) * c2 > RefMax<F8>::kLazy) {
-            const float neg_new = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
-            l_run *= fast_exp2(__fsub_rn(neg_new, neg));      // the helper derives the same factor from the same two values
-            m_ref = mxa;
-            neg = neg_new;
-          }
-          s_neg[i * 128 + row] = neg;
-          mbar_arrive(&row_ready[i]);
-          SDVG_TRACE(i, 3000 + j);
-          // ---- P = 2^(c2 * (S - m_ref)), bf16, written back over S: columns 0-63, then 64-95 ------
-          const uint64_t negx2 = pack2(neg, neg);
-          uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
-          uint32_t pk[F8 ? 8 : 16];
-          if constexpr (F8) {
-            exp_chunk_f8(s[0], c2x2, negx2, pk, sum_a, sum_b);
-            tmem_st8(tS, pk);
-            exp_chunk_f8(s[1], c2x2, negx2, pk, sum_a, sum_b);
-            tmem_st8(tS + 8, pk);
-          } else {
-            exp_chunk(s[0], c2x2, negx2, pk, sum_a, sum_b);
-            tmem_st16(tS, pk);
-            exp_chunk(s[1], c2x2, negx2, pk, sum_a, sum_b);
-            tmem_st16(tS + 16, pk);
-          }
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&p_lo[i]);
-          SDVG_TRACE(i, 4000 + j);
-          if constexpr (F8) {
-            exp_chunk_f8(s[2], c2x2, negx2, pk, sum_a, sum_b);
-            tmem_st8(tS + 16, pk);
-          } else {
-            exp_chunk(s[2], c2x2, negx2, pk, sum_a, sum_b);
-            tmem_st16(tS + 32, pk);
-          }
-          {
-            float a0, a1, b0, b1;
-            unpack2(sum_a, a0, a1);
-            unpack2(sum_b, b0, b1);
-            l_run += (a0 + a1) + (b0 + b1);
-          }
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&p_mid[i]);
-          SDVG_TRACE(i, 5000 + j);
+      #pragma unroll 1
+      for (int j = 0; j < my_nk && alive; ++j) {          // this lane's j-th key tile
+        // number of real keys in that tile: the last tile of a key segment may be ragged
+        const int valid = key_tile_valid(p, it.key_tile(i, j));
+        const uint32_t par = s_cnt & 1;
+        SDVG_TRACE(i + 3 * half, 0 + j);
+        if (!(alive = wait_bar(&s_full[i], par, dl))) break;
+        SDVG_TRACE(i + 3 * half, 1000 + j);
+        tc_fence_after();
+        // ---- this thread's 64 logits of the row into registers; S is then free for the other lane's product
+        uint32_t s[2][32];
+        tmem_ld32(tS, s[0]);
+        tmem_ld32(tS + 32, s[1]);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(s_free);
+        if (valid < kTileN) {
+          // ragged last tile of a key segment (TMA zero-filled the missing keys): their logits become -inf
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+              if (half * 64 + c * 32 + k >= valid) s[c][k] = 0xff800000u;
         }
+        // ---- row maximum: own half, published for the row's other thread
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        max_chunk(s[0], mx);
+        max_chunk(s[1], mx);
+        const float mx_own = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        my_max[par * 512] = mx_own;
+        mbar_arrive(&mx_ready[i]);
+        SDVG_TRACE(i + 3 * half, 2000 + j);
+        if (!(alive = wait_bar(&mx_ready[i], par, dl))) break;
+        const float mxa = fmaxf(mx_own, other_max[par * 512]);
+        // both threads of the row take the same decision from the same values
+        float alpha = 1.f;
+        bool moved = false;
+        if (j == 0) {
+          m_ref = mxa;
+          neg = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
+        } else if ((mxa - m_ref) * c2 > RefMax<F8>::kLazy) {
+          const float neg_new = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
+          alpha = fast_exp2(__fsub_rn(neg_new, neg));
+          l_run *= alpha;
+          m_ref = mxa;
+          neg = neg_new;
+          moved = true;
+        }
+        SDVG_TRACE(i + 3 * half, 3000 + j);
+        if (__any_sync(0xffffffffu, moved)) {
+          // Rare: the reference maximum of a row moved, so what O_i holds of that row is rescaled before the
+          // next product adds to it; each of the row's two threads takes half of the head dimension.
+          // PV_i(j-1) is commit number s_cnt - 1 on o_full[i].
+          if (!(alive = wait_bar(&o_full[i], (s_cnt - 1) & 1, dl))) break;
+          tc_fence_after();
+          if ((tid & 31) == 0) atomicAdd(p.work + 2, 1u);      // diagnostic count of warp-level rescale events
+#pragma unroll 1
+          for (int c = 0; c < D / 64; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + half * (D / 2) + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
+            tmem_st32(tO + half * (D / 2) + c * 32, o);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+        // ---- P = 2^(c2 * (S - m_ref)) for this thread's 64 keys
+        const uint64_t negx2 = pack2(neg, neg);
+        uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
+        uint32_t pk0[F8 ? 8 : 16], pk1[F8 ? 8 : 16];
+        if constexpr (F8) {
+          if (half == 0) {
+            exp_chunk_f8<Mix::kSoftmax>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk_f8<Mix::kSoftmax>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+          } else {
+            exp_chunk_f8<Mix::kHelper>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk_f8<Mix::kHelper>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+          }
+        } else {
+          if (half == 0) {
+            exp_chunk<Mix::kSoftmax>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk<Mix::kSoftmax>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+          } else {
+            exp_chunk<Mix::kHelper>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk<Mix::kHelper>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+          }
+        }
+        {
+          float a0, a1, b0, b1;
+          unpack2(sum_a, a0, a1);
+          unpack2(sum_b, b0, b1);
+          l_run += (a0 + a1) + (b0 + b1);
+        }
+        // the previous P of this lane must have been consumed: its product is commit number s_cnt - 1 on o_full
+        if (s_cnt > 0) {
+          if (!(alive = wait_bar(&o_full[i], (s_cnt - 1) & 1, dl))) break;
+          tc_fence_after();
+        }
+        ++s_cnt;
+        if constexpr (F8) {
+          tmem_st8(tP, pk0);
+          tmem_st8(tP + 8, pk1);
+        } else {
+          tmem_st16(tP, pk0);
+          tmem_st16(tP + 16, pk1);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&p_ready[i]);
+        SDVG_TRACE(i + 3 * half, 4000 + j);
       }
       if (!alive) break;
-      // ---- epilogue: add the helper's share of the row sum, wait for the last PV, normalise, store
-      // (the next item's first arrival on p_lo comes after these TMEM reads, which is what lets the
-      // issuer overwrite O_i then)
-      if (!(alive = wait_bar(&l_ready[i], item_cnt & 1, dl))) break;
+      // ---- epilogue: the lower-half thread of a row adds the upper half's share of the row sum, waits for
+      // the last product, normalises and stores the row (the next item's first arrival on p_ready comes
+      // after these TMEM reads, which is what lets the issuer overwrite O_i then)
+      if (half == 1) {
+        s_rowsum[i * 128 + row] = l_run;
+        mbar_arrive(&sum_ready[i]);
+        if (it.split && i == 1) {                        // lane 1 of a split tile: O_1 is read by lane 0's threads
+          alive = wait_bar(merge_done, split_cnt & 1, dl);
+          ++split_cnt;
+        }
+        continue;
+      }
+      if (!(alive = wait_bar(&sum_ready[i], item_cnt & 1, dl))) break;
       ++item_cnt;
-      l_run += s_lhelp[i * 128 + row];
+      l_run += s_rowsum[i * 128 + row];
       pv_cnt += my_nk;
       if (!(alive = wait_bar(&o_full[i], (pv_cnt - 1) & 1, dl))) break;
       tc_fence_after();
@@ -826,20 +779,20 @@ __global__ void __launch_bounds__(512, 1) attn_fwd_ws_kernel(const __grid_consta
       // own reference maximum.  Lane 1 publishes (-m*c2, l) and waits until lane 0 has folded O_1 into its output.
       float w0 = 1.f, w1 = 0.f;                      // weights of O_0 and O_1 in the merged numerator
       if (it.split) {
-        const uint32_t par = split_cnt & 1;
+        const uint32_t spar = split_cnt & 1;
         ++split_cnt;
         if (i == 1) {
           s_merge[row] = neg;
-          s_neg[128 + row] = l_run;
+          s_merge[128 + row] = l_run;
           tc_fence_before();
           mbar_arrive(lane1_done);
-          alive = wait_bar(merge_done, par, dl);
+          alive = wait_bar(merge_done, spar, dl);
           if (!alive) break;
           continue;
         }
-        if (!(alive = wait_bar(lane1_done, par, dl))) break;
+        if (!(alive = wait_bar(lane1_done, spar, dl))) break;
         tc_fence_after();
-        const float neg1 = s_merge[row], l1 = s_neg[128 + row];
+        const float neg1 = s_merge[row], l1 = s_merge[128 + row];
         const float negm = fminf(neg, neg1);         // the larger of the two reference maxima
         w0 = fast_exp2(negm - neg);                  // 2^((m_0 - m) c2) <= 1: rebases lane 0's sums to the common maximum
         w1 = fast_exp2(negm - neg1);

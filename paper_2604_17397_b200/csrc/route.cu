@@ -64,16 +64,24 @@ __device__ __forceinline__ long long range_begin(const RouteParams& p, int b) {
   return p.offsets ? (long long)p.offsets[b] : (long long)b * p.frames_per_block;
 }
 
+// The offsets live in device memory, so the host cannot check them.  The kernel trusts only the two ends of the
+// array: every read stays inside [offsets[0], offsets[num_blocks]), and a block whose own range leaves that
+// interval or runs backwards counts as a block without frames (accept 0, NaN aggregate, argmin -1).
+__device__ __forceinline__ bool range_ok(long long s, long long e, long long all_lo, long long all_hi) {
+  return all_lo <= s && s <= e && e <= all_hi;
+}
+
 __global__ void __launch_bounds__(kThreads) route_kernel(const __grid_constant__ RouteParams p) {
   __shared__ __align__(16) float stage[kSmemFloats + 4];   // +4: room for the alignment shift
   const int ntiles = (p.num_blocks + kThreads - 1) / kThreads;
+  const long long all_lo = range_begin(p, 0), all_hi = range_begin(p, p.num_blocks);
   for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int b0 = tile * kThreads;
     const int b1 = min(b0 + kThreads, p.num_blocks);
     const long long lo = range_begin(p, b0);
     const long long hi = range_begin(p, b1);
     const long long n = hi - lo;
-    const bool staged = n > 0 && n <= kSmemFloats;
+    const bool staged = n > 0 && n <= kSmemFloats && range_ok(lo, hi, all_lo, all_hi);
     if (staged) {
       // stage[i] = scores[lo + i]; vector body starts at the first 16-byte aligned element
       const float* src = p.scores + lo;
@@ -91,18 +99,25 @@ __global__ void __launch_bounds__(kThreads) route_kernel(const __grid_constant__
       __syncthreads();
       const int b = b0 + threadIdx.x;
       if (b < b1) {
-        const int s = (int)(range_begin(p, b) - lo) + shift;
-        const int e = (int)(range_begin(p, b + 1) - lo) + shift;
+        long long s = range_begin(p, b), e = range_begin(p, b + 1);
+        if (!range_ok(s, e, all_lo, all_hi)) e = s;          // malformed: no frames
         float m;
         int idx;
-        aggregate(p, s, e, [&](long long i) { return stage[i]; }, m, idx);
+        if (lo <= s && e <= hi) {
+          const int sh = shift - (int)lo;
+          aggregate(p, s, e, [&](long long i) { return stage[i + sh]; }, m, idx);
+        } else {
+          // offsets that are not sorted can place a block outside its tile's range: read it where it is
+          aggregate(p, s, e, [&](long long i) { return p.scores[i]; }, m, idx);
+        }
         decide(p, b, m, idx, e > s);
       }
       __syncthreads();
     } else {
       const int b = b0 + threadIdx.x;
       if (b < b1) {
-        const long long s = range_begin(p, b), e = range_begin(p, b + 1);
+        long long s = range_begin(p, b), e = range_begin(p, b + 1);
+        if (!range_ok(s, e, all_lo, all_hi)) e = s;          // malformed: no frames
         float m;
         int idx;
         aggregate(p, s, e, [&](long long i) { return p.scores[i]; }, m, idx);

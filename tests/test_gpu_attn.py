@@ -232,23 +232,39 @@ def test_bounded_wait_gives_up_reports_timeout_and_leaves_the_context_usable():
     dt = time.perf_counter() - t0
     assert 0.015 <= dt < 1.0, dt
     assert int(ws.view(torch.int32)[0].item()) == 2                  # the waiting warp ran to its end
-    # the device still works: a normal attention call on the same workspace succeeds and clears the status
+    # the device still works: a normal attention call on the same workspace succeeds; the status word is
+    # sticky, so the timeout stays visible until the workspace is reset
     sh = synth.TINY
     cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
     q, k, v = (to_dev(synth.block_tensor(sh, 80, 0, 0, t)) for t in (synth.Q, synth.K, synth.V))
-    out = torch.empty_like(q)
+    out = torch.full_like(q, float("nan"))
+    api.sdvg_block_attn_fwd(q, k, v, cache, 0, out, None, sh.scale, ws)
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_ERR_TIMEOUT
+    assert torch.isfinite(out.float()).all()
+    api.sdvg_block_attn_workspace_reset(ws)
     api.sdvg_block_attn_fwd(q, k, v, cache, 0, out, None, sh.scale, ws)
     assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
-    assert torch.isfinite(out.float()).all()
+
+
+def _lazy_raises(tile_max_log2, lazy=8.0):
+    """Number of times the lazy reference-maximum policy moves the reference of a row, given the row's
+    per-key-tile maxima in the exp2 domain, in the order a lane visits the tiles: the first tile sets the
+    reference, a later tile moves it when its maximum exceeds it by more than 2^lazy."""
+    ref, n = tile_max_log2[0], 0
+    for m in tile_max_log2[1:]:
+        if m - ref > lazy:
+            ref, n = m, n + 1
+    return n
 
 
 def test_rising_logits_rescale_the_accumulator_at_almost_every_key_tile():
     # Keys whose magnitude grows along the sequence: the row maximum keeps rising by more than the lazy-rescale
-    # threshold, so the helper warps rescale O (and both partial row sums) again and again.
+    # threshold, so the softmax threads rescale O (and their partial row sums) again and again.
     sh = synth.Shape("rising", heads=2, head_dim=128, frames=3, grid_h=16, grid_w=16, slots=3)   # 768 tokens = 6 key tiles per block
     cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
     ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
     ws = api.attn_workspace()
+    ks = []
     for b in range(3):
         q = synth.block_tensor(sh, 90, b, 0, synth.Q, std=1.0)
         # all queries share a direction with the keys so that logits grow with the key index
@@ -257,17 +273,32 @@ def test_rising_logits_rescale_the_accumulator_at_almost_every_key_tile():
         k = O.f64_to_bf16(base * ramp + 0.05 * O.bf16_to_f64(synth.block_tensor(sh, 90, b, 0, synth.K)))
         q = O.f64_to_bf16(np.abs(O.bf16_to_f64(q)) * np.sign(base) * 1.5)
         v = synth.block_tensor(sh, 90, b, 0, synth.V)
+        ks.append(k)
         dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
         out = torch.full_like(dq, float("nan"))
         lse = torch.full((sh.heads, sh.block_tokens), float("nan"), device="cuda")
         api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_STAGE)
+        api.sdvg_block_attn_workspace_reset(ws)
         api.sdvg_block_attn_fwd(dq, None, None, cache, b, out, lse, sh.scale, ws)
         assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
         o_ref, lse_ref = O.block_attn_ref(q, k, v, ref, b, sh.scale)
-        # the logits of one row span far more than 2^8 between the first and the last key tile
-        assert (lse_ref.max() - lse_ref.min()) >= 0 and np.isfinite(lse_ref).all()
         check(to_bits(out), o_ref, ("rising", b))
         assert np.allclose(lse.cpu().numpy(), lse_ref, rtol=2e-4, atol=2e-3)
+        # The rescale path must have run.  From the exact logits: how often does the lazy policy move a row's
+        # reference, whether a lane visits every key tile or every second one (a query tile that is worked on by
+        # both lanes)?  A warp takes the path when any of its 32 rows moves, and a row has two threads, in two warps.
+        kk = np.concatenate([O.bf16_to_f64(x) for x in ks], axis=0)                  # keys in ring order (no wrap yet)
+        logit2 = np.einsum("thd,shd->hts", O.bf16_to_f64(q), kk) * sh.scale * 1.4426950408889634
+        tile_max = logit2.reshape(sh.heads, sh.block_tokens, -1, 128).max(axis=3)    # [heads, rows, key tiles]
+        floor_events = 0
+        for h in range(sh.heads):
+            per_row = np.array([min(_lazy_raises(tile_max[h, r]), _lazy_raises(tile_max[h, r, 0::2]) +
+                                    _lazy_raises(tile_max[h, r, 1::2])) if tile_max.shape[2] > 1 else 0
+                                for r in range(sh.block_tokens)])
+            floor_events += 2 * int(per_row.reshape(-1, 32).min(axis=1).sum())
+        events = api.sdvg_block_attn_rescale_events(ws)
+        assert floor_events >= 2 * sh.heads * (sh.block_tokens // 32), floor_events       # the data does force it
+        assert events >= floor_events, (events, floor_events)
         api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_FINAL)
         ref.commit(b, k, v, O.FINAL)
 
