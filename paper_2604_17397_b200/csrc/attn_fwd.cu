@@ -341,11 +341,6 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kWorkspaceBytes
 
 extern "C" {
 
-#ifdef SDVG_ATTN_TRACE
-// Developer build only: device buffer of [6][512][2] int64 that CTA 0 fills with (event, clock) pairs.
-int sdvg_debug_set_trace(void* p) { return (int)cudaMemcpyToSymbol(g_trace, &p, sizeof(p)); }
-#endif
-
 size_t sdvg_block_attn_workspace_bytes(void) { return kWorkspaceBytes; }
 
 int sdvg_block_attn_workspace_reset(void* workspace, size_t workspace_bytes, void* stream_) {

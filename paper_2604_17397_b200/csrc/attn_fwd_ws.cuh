@@ -1,70 +1,50 @@
 // Warp-specialised, persistent block-attention kernel (included by attn_fwd.cu after the common
-// definitions).  One CTA per SM; a work item is a pair of 128-row query tiles ("lanes").  Usually
-// the two tiles belong to one head and share every K/V tile; a pair that straddles a head boundary
-// has lanes that stream their own K/V, and the tiles left over after the pairs run alone.
+// definitions).  One CTA of 20 warps per SM; a work item is a pair of 128-row query tiles ("lanes").
+// Usually the two tiles belong to one head and share every K/V tile; a pair that straddles a head
+// boundary has lanes that stream their own K/V, and the tiles left over after the pairs run alone,
+// their keys split between the two lanes.
 //
-//   warps 0-3   softmax of lane 0 (one thread per row)            \  S, P and O live in tensor memory:
-//   warps 4-7   softmax of lane 1                                  >  S0 S1 O0 O1 = 4 x 128 columns
-//   warps 8-11  helper: rescales O when a row maximum moved, and  /
-//               exponentiates the last 32 key columns of both lanes
-//   warp  12    TMA producer: Q tiles, then the K/V ring
-//   warp  13    MMA issuer: S_i = Q_i K^T, O_i += P_i V
-//   warps 14-15 idle
+//   warps 0-3    softmax of lane 0, key columns 0-63 of every tile     \  two threads per query row: a warp
+//   warps 4-7    softmax of lane 1, key columns 0-63                    \ reaches the 32 TMEM lanes of its place
+//   warps 8-11   softmax of lane 0, key columns 64-127                  / in its warpgroup, so the threads of a
+//   warps 12-15  softmax of lane 1, key columns 64-127                 /  row sit in warps w and w + 8
+//   warp  16     TMA producer: Q tiles, then the K/V ring
+//   warp  17     MMA issuer of the first product,  S = Q_i K^T
+//   warp  18     MMA issuer of the second product, O_i += P_i V
+//   warp  19     idle (warps come in fours: one per SM sub-partition)
 //
-// Tensor-pipe order per key tile j:  PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1); while the pipe works for
-// lane 1 the softmax warps of lane 0 turn S_0(j+1) into P_0(j+1), and vice versa.  The running row
-// maximum is only raised when it grew by more than 2^8 in the exp2 domain, so O is rarely rescaled
-// and that work stays off the critical path; the final 1/l normalisation and the store are done by
-// the softmax warps themselves, which own the same TMEM lanes.
+// Tensor memory: O_0 and O_1 (128 columns each), ONE S (128 columns) that the lanes use in turn, P_0 and P_1
+// (64 columns each: bf16 pairs).  S only lives from the end of its product until the softmax threads of its
+// lane have read it into registers (s_free); the first product of the NEXT key tile of the other lane can
+// then start, whatever the softmax of either lane is doing.  Each lane's first product therefore runs one
+// key tile ahead of its softmax, and the chain "S ready -> softmax -> P ready -> second product -> next
+// first product -> S ready" that would otherwise pace a lane is cut: the softmax threads find their next row
+// of S waiting when they have stored P, and the second product only has to finish before the lane's NEXT P
+// is stored (o_full).  What paces the kernel is then the slower of the tensor pipe and the special-function
+// unit: a 128 x 128 tile needs 16384 exponentials at 16 per clock per SM, the same 1024 clocks its two
+// products take.
 //
-// The chain S ready -> softmax -> P ready -> PV, QK -> next S ready of one lane sets the pace, so it
-// is shortened from both ends.  A softmax thread reduces its whole row of S to the maximum, hands
-// the reference maximum to the helper thread of the same row, and exponentiates key columns 0-95;
-// the helper thread does columns 96-127 meanwhile.  P is released to the issuer in two parts
-// (columns 0-63 and 96-127 together with "O rescaled", then columns 64-95), and the issuer starts
-// the PV product on the first part while the softmax thread finishes the third quarter.  The issuer
-// is blocked while the tensor pipe's queue is full, so it looks at the K/V stages of its next step
-// right after queueing a batch of MMAs, when that costs nothing.  The producer and issuer warps
-// run their loops with all 32 lanes (warp-uniform control flow and values) and only predicate the
-// TMA / MMA / commit instructions on one elected lane: descriptors and addresses then stay in
-// uniform registers.  All role loops are kept small (rare paths rolled, ragged tiles masked in
-// tensor memory by a cold loop): the roles share the SM's instruction cache, and the issuer, which
-// runs once per key tile, pays for every line the others push out.
+// A softmax thread reads its 64 logits, reduces them to a maximum, swaps that with the row's other thread
+// through shared memory (mx_ready), and both take the same decision: the reference maximum m is only
+// raised when the row maximum outgrew it by more than 2^8 in the exp2 domain, so O is rarely rescaled
+// (when it is, each of the two threads rescales half of the head dimension).  P = 2^(c S - c m) is
+// rounded to bf16 and stored to the lane's P columns; the row sum is kept per thread and added up when the
+// item ends, where the lower-half thread normalises by 1/l and stores the row.
+// The two products have an issuing warp each, so that the waits and bookkeeping of one overlap the MMAs
+// of the other (the tensor pipe queues only a few instructions).  The producer and issuer warps run their
+// loops with all 32 lanes (warp-uniform control flow and values) and only predicate the TMA / MMA / commit
+// instructions on one elected lane: descriptors and addresses then stay in uniform registers.
 //
-// The exponentials are the co-limiter of this kernel: a 128 x 128 tile needs 16384 of them and the
-// special-function unit delivers 16 per clock per SM, the same 1024 clocks the tile's two MMAs take.
-// A compile-time share of the elements can be evaluated on the FMA pipe instead (range reduction to
-// [0, 1) plus a cubic, relative error 2e-4, a tenth of the bf16 rounding P gets anyway); it is off by
-// default (SDVG_ATTN_POLY_PAIRS = 0) because the extra instructions cost more than the freed
-// special-function slots gain once the GPU runs under its power cap.
+// A compile-time share of the exponentials can be evaluated on the FMA pipe instead (range reduction to
+// [0, 1) plus a cubic, relative error 2e-4, a tenth of the bf16 rounding P gets anyway); it is off because
+// the extra instructions cost more issue slots than the freed special-function slots gain.
 //
 // 8-bit variant (template flag F8): Q, K and V tiles are E4M3 bytes (a 128-dim row is one 128-byte panel, so a
 // tile is half the size and the ring holds 8 stages), both products use the 8-bit MMA kind (K = 32 per
 // instruction, half the tensor-pipe time), P is rounded to E4M3 (four per TMEM column) and the per-head
-// scales enter as a factor of the logit scale and of the final 1/l.  Everything else (roles, barriers,
-// schedule, lazy maximum, split tiles) is shared; the softmax, not the tensor pipe, then sets the pace.
+// scales enter as a factor of the logit scale and of the final 1/l.  Everything else is shared.
 #pragma once
 
-#ifdef SDVG_ATTN_TRACE
-__device__ long long* g_trace = nullptr;     // [6 roles][512 events][id, clock]
-#define SDVG_TRACE_DECL(cond)                 \
-  long long* const tr_base = g_trace;         \
-  const bool tr_on = (cond) && tr_base;       \
-  int tr_n = 0;
-#define SDVG_TRACE(role, id)                                                                      \
-  do {                                                                                            \
-    if (tr_on && tr_n < 512) {                                                                    \
-      longlong2 ev_;                                                                              \
-      ev_.x = (id);                                                                               \
-      ev_.y = clock64();                                                                          \
-      reinterpret_cast<longlong2*>(tr_base)[(role)*512 + tr_n] = ev_;                             \
-      ++tr_n;                                                                                     \
-    }                                                                                             \
-  } while (0)
-#else
-#define SDVG_TRACE_DECL(cond)
-#define SDVG_TRACE(role, id) do { } while (0)
-#endif
 
 // F8: operands are E4M3 bytes instead of bf16 (a row of 128 dims is then one 128-byte panel).
 template <int D, bool F8 = false>
@@ -221,31 +201,25 @@ __device__ __forceinline__ void exp2_poly2(uint64_t x2, float& e0, float& e1) {
   e1 = __uint_as_float(__float_as_uint(t1) * 0x00800000u + __float_as_uint(p1));
 }
 
-// Share of the exponentials that goes to the FMA pipe, per role: out of every 4 consecutive element pairs
-// of a 32-column chunk this many take the polynomial (4 = the whole chunk).
-#ifndef SDVG_MIX_HELPER
-#define SDVG_MIX_HELPER 0
+// Share of the exponentials that goes to the FMA pipe: out of every 4 consecutive element pairs of a
+// 32-column chunk this many take the polynomial (4 = the whole chunk), separately for the threads that own
+// key columns 0-63 and 64-127 of a row.
+#ifndef SDVG_POLY_LOWER
+#define SDVG_POLY_LOWER 0
 #endif
-#ifndef SDVG_MIX_SOFTMAX
-#define SDVG_MIX_SOFTMAX 0
+#ifndef SDVG_POLY_UPPER
+#define SDVG_POLY_UPPER 0
 #endif
-#ifndef SDVG_MIX_SOFTMAX_MID
-#define SDVG_MIX_SOFTMAX_MID 0
+#ifndef SDVG_POLY_LOWER_F8
+#define SDVG_POLY_LOWER_F8 0
 #endif
-#ifndef SDVG_MIX_HELPER_F8
-#define SDVG_MIX_HELPER_F8 0
-#endif
-#ifndef SDVG_MIX_SOFTMAX_F8
-#define SDVG_MIX_SOFTMAX_F8 0
-#endif
-#ifndef SDVG_MIX_SOFTMAX_MID_F8
-#define SDVG_MIX_SOFTMAX_MID_F8 0
+#ifndef SDVG_POLY_UPPER_F8
+#define SDVG_POLY_UPPER_F8 0
 #endif
 template <bool F8>
 struct ExpMix {
-  static constexpr int kHelper = F8 ? SDVG_MIX_HELPER_F8 : SDVG_MIX_HELPER;            // key columns 96-127
-  static constexpr int kSoftmax = F8 ? SDVG_MIX_SOFTMAX_F8 : SDVG_MIX_SOFTMAX;         // key columns 0-63
-  static constexpr int kSoftmaxMid = F8 ? SDVG_MIX_SOFTMAX_MID_F8 : SDVG_MIX_SOFTMAX_MID;   // key columns 64-95
+  static constexpr int kLower = F8 ? SDVG_POLY_LOWER_F8 : SDVG_POLY_LOWER;     // key columns 0-63
+  static constexpr int kUpper = F8 ? SDVG_POLY_UPPER_F8 : SDVG_POLY_UPPER;     // key columns 64-127
 };
 
 // One 32-column chunk of a row: P = 2^(c2 * S - m*c2) as bf16 pairs, returns the packed partial row sums.
@@ -408,7 +382,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       uint32_t q_cnt[2] = {0, 0}, kv_issued = 0;
       RingPos ring;
       bool alive = true;
-      SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
 
       // one K or V tile of key tile j of `head` into the next ring stage
       auto load_kv = [&](bool is_v, int head, int j) {
@@ -419,7 +392,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
           kt -= nt;
         }
         if (!(alive = wait_warp(&kv_empty[ring.stage], ring.phase ^ 1, dl))) return;
-        SDVG_TRACE(4, kv_issued);
         if (leader) {
           mbar_expect_tx(&kv_full[ring.stage], C::kTileBytes);
           const AttnProblem& pr = p.prob[head / p.heads];
@@ -477,7 +449,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       uint32_t qk_cnt = 0;                 // products written into S so far = phase index of s_free
       RingPos ring;                        // walks every entry of the K/V ring; this warp consumes the K tiles
       bool alive = true;
-      SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
       // Descriptors of stage 0 and of the two query tiles, built once; a stage or a 16-wide slice is then one
       // addition to the address field (all of this CTA's shared memory fits that field, so nothing carries out).
       const uint64_t descQ0 = smem_desc_sw128(sQ, 16, 1024);
@@ -493,7 +464,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         }
         if (qk_cnt > 0 && !(alive = wait_warp(s_free, (qk_cnt - 1) & 1, dl))) return;
         ++qk_cnt;
-        SDVG_TRACE(2, 50000 + i * 1000);
         tc_fence_after();
         if (leader) {
           const uint32_t d = tmem_base + kColS;
@@ -513,7 +483,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
           if (release_stage) mma_commit(&kv_empty[st]);
           if (last_of_item) mma_commit(&q_empty[i]);
         }
-        SDVG_TRACE(2, 60000 + i * 1000);
       };
 
       #pragma unroll 1
@@ -556,7 +525,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       uint32_t pv_par = 0;                 // bit i: phase parity of lane i's P barrier
       RingPos ring;                        // walks every entry of the K/V ring; this warp consumes the V tiles
       bool alive = true;
-      SDVG_TRACE_DECL(blockIdx.x == 0 && leader)
       const uint64_t descV0 = smem_desc_sw128(sKV, C::kPanelBytes, 1024);
       constexpr int kSlices = F8 ? 4 : 8;  // MMAs per key tile: 32 or 16 keys each
 
@@ -587,7 +555,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
             // P_i stored and O_i rescaled where a row maximum moved (for t = 0: O_i was read out by the
             // epilogue of the previous item before its softmax threads arrived here)
             if (!(alive = wait_warp(&p_ready[i], par, dl))) break;
-            SDVG_TRACE(5, 3000 + i * 1000 + t);
             tc_fence_after();
             if (leader) {
               // O_i (+)= P_i[:, slice kk] V[slice kk, :]; slice kk of P is 8 TMEM columns (16 bf16 or 32 bytes per
@@ -604,7 +571,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
               mma_commit(&o_full[i]);
               if (last_user) mma_commit(&kv_empty[stV]);
             }
-            SDVG_TRACE(5, 9000 + i * 1000 + t);
           }
         }
       }
@@ -628,7 +594,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
     uint64_t c2x2 = pack2(c2, c2);
     uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0, split_cnt = 0;
     bool alive = true;
-    SDVG_TRACE_DECL(blockIdx.x == 0 && row == 0 && (half == 0 || i == 0))
     #pragma unroll 1
     for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
       WsItem it;
@@ -648,9 +613,7 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         // number of real keys in that tile: the last tile of a key segment may be ragged
         const int valid = key_tile_valid(p, it.key_tile(i, j));
         const uint32_t par = s_cnt & 1;
-        SDVG_TRACE(i + 3 * half, 0 + j);
         if (!(alive = wait_bar(&s_full[i], par, dl))) break;
-        SDVG_TRACE(i + 3 * half, 1000 + j);
         tc_fence_after();
         // ---- this thread's 64 logits of the row into registers; S is then free for the other lane's product
         uint32_t s[2][32];
@@ -674,7 +637,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         const float mx_own = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         my_max[par * 512] = mx_own;
         mbar_arrive(&mx_ready[i]);
-        SDVG_TRACE(i + 3 * half, 2000 + j);
         if (!(alive = wait_bar(&mx_ready[i], par, dl))) break;
         const float mxa = fmaxf(mx_own, other_max[par * 512]);
         // both threads of the row take the same decision from the same values
@@ -691,7 +653,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
           neg = neg_new;
           moved = true;
         }
-        SDVG_TRACE(i + 3 * half, 3000 + j);
         if (__any_sync(0xffffffffu, moved)) {
           // Rare: the reference maximum of a row moved, so what O_i holds of that row is rescaled before the
           // next product adds to it; each of the row's two threads takes half of the head dimension.
@@ -717,19 +678,19 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         uint32_t pk0[F8 ? 8 : 16], pk1[F8 ? 8 : 16];
         if constexpr (F8) {
           if (half == 0) {
-            exp_chunk_f8<Mix::kSoftmax>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
-            exp_chunk_f8<Mix::kSoftmax>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+            exp_chunk_f8<Mix::kLower>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk_f8<Mix::kLower>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
           } else {
-            exp_chunk_f8<Mix::kHelper>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
-            exp_chunk_f8<Mix::kHelper>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+            exp_chunk_f8<Mix::kUpper>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk_f8<Mix::kUpper>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
           }
         } else {
           if (half == 0) {
-            exp_chunk<Mix::kSoftmax>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
-            exp_chunk<Mix::kSoftmax>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+            exp_chunk<Mix::kLower>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk<Mix::kLower>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
           } else {
-            exp_chunk<Mix::kHelper>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
-            exp_chunk<Mix::kHelper>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
+            exp_chunk<Mix::kUpper>(s[0], c2x2, negx2, pk0, sum_a, sum_b);
+            exp_chunk<Mix::kUpper>(s[1], c2x2, negx2, pk1, sum_a, sum_b);
           }
         }
         {
@@ -754,7 +715,6 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&p_ready[i]);
-        SDVG_TRACE(i + 3 * half, 4000 + j);
       }
       if (!alive) break;
       // ---- epilogue: the lower-half thread of a row adds the upper half's share of the row sum, waits for

@@ -45,3 +45,29 @@ def test_single_rank_passthrough():
     dist_util.barrier(1)
     with pytest.raises(ValueError):
         dist_util.shard_heads(12, 8, 0)
+
+
+def test_bench_gpus_flag_spawns_that_many_ranks():
+    # `bench.py --gpus 2` run without a launcher's environment must start two ranks itself; --plumbing-only makes
+    # the ranks meet over gloo and report their places instead of touching a GPU
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--plumbing-only"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                    # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["gpus_requested"] == 2
+    assert [p["rank"] for p in line["places"]] == [0, 1]
+    assert [p["local_rank"] for p in line["places"]] == [0, 1]
+    assert line["places"][0]["pid"] != line["places"][1]["pid"]
+    assert line["max_over_ranks"] == 2.0
+
+
+def test_spawner_refuses_zero_ranks():
+    with pytest.raises(ValueError):
+        dist_util.spawn_ranks(0, ["x.py"])
