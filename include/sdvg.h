@@ -410,6 +410,39 @@ int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_
                              int64_t block_index, const float* qk_descale, const float* v_descale, void* out,
                              float* lse, float scale, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- the denoising steps of a block in one call ------------------------------- */
+/*
+ * Sec. 4.1 "Models": each block takes 4 denoising steps; Sec. 3 "Inference flow": the drafter pays them for
+ * every block and the target for every rejected one.  This call enqueues, for s = 0 .. steps-1 and in order,
+ *   sdvg_rope3d_qk_commit(cache, q[s], k[s], v[s], q_roped[s], NULL, ..., block_index, SDVG_STAGE)
+ *   sdvg_block_attn_fwd(q_roped[s], NULL, NULL, cache, block_index, out[s], NULL, scale, workspace)
+ * on `stream`: 2 * steps kernels, nothing else.  The ring state does not change (SDVG_STAGE), so the block's
+ * final commit still follows.  The results are those of the separate calls, bit for bit.
+ *   q, k, v, q_roped, out   HOST arrays of `steps` device pointers (bf16 [block_tokens, heads, head_dim] each;
+ *                           the arrays are read during the call only)
+ *   steps                   1 .. 64
+ * Every pointer, the workspace, the scale and the block index are checked for all steps before the first
+ * launch; grid, table and device are checked by the first prologue, before it launches.
+ * Errors: those of the two calls; BAD_SHAPE also for steps outside 1 .. 64 or an 8-bit ring.
+ */
+int sdvg_block_steps(int steps, sdvg_cache* cache, const void* const* q, const void* const* k,
+                     const void* const* v, void* const* q_roped, void* const* out,
+                     int frames, int grid_h, int grid_w, int frame_offset,
+                     const float* cos_sin_tab, int tab_frames, int64_t block_index, float scale,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same for an 8-bit ring: sdvg_rope3d_qk_commit_e4m3 (q8_roped[s] receives E4M3 codes, device bytes
+ * [block_tokens, heads, 128]) followed by sdvg_block_attn_fwd_e4m3, with the scale vectors of those calls.
+ */
+int sdvg_block_steps_e4m3(int steps, sdvg_cache* cache, const void* const* q, const void* const* k,
+                          const void* const* v, void* const* q8_roped, void* const* out,
+                          const float* q_inv_scale, const float* k_inv_scale, const float* v_inv_scale,
+                          const float* qk_descale, const float* v_descale,
+                          int frames, int grid_h, int grid_w, int frame_offset,
+                          const float* cos_sin_tab, int tab_frames, int64_t block_index, float scale,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

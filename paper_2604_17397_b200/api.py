@@ -69,6 +69,9 @@ SIGNATURES = {
     "sdvg_rope3d_qk_commit_e4m3": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
                                         C.POINTER(_I64), _VP]),
     "sdvg_block_attn_fwd_e4m3": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
+    "sdvg_block_steps": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _F, _VP, _SZ, _VP]),
+    "sdvg_block_steps_e4m3": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I,
+                                   _I64, _F, _VP, _SZ, _VP]),
 }
 
 _lib = None
@@ -449,3 +452,42 @@ def sdvg_block_attn_fwd_e4m3(q8, k_self8, v_self8, cache: Cache, block_index: in
                                         _bf16(out, shape), _ptr(lse), scale, workspace.data_ptr(), workspace.numel(),
                                         _stream(stream))
     _check(st, "sdvg_block_attn_fwd_e4m3")
+
+
+# ---------------------------------------------------------------- the steps of a block in one call
+
+def _ptr_array(ts, check):
+    return (_VP * len(ts))(*[check(t) for t in ts])
+
+
+def sdvg_block_steps(cache: Cache, qs, ks, vs, q_ropeds, outs, grid, frame_offset: int, table, tab_frames: int,
+                     block_index: int, scale: float, workspace: torch.Tensor, stream=None) -> None:
+    """The denoising steps of one block (lists of per-step tensors): fused rope + stage, then attention, per step."""
+    n = len(qs)
+    if not (len(ks) == len(vs) == len(q_ropeds) == len(outs) == n):
+        raise ValueError("one q, k, v, q_roped and out per step")
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    bf = lambda t: _bf16(t, shape)
+    arrays = [_ptr_array(x, bf) for x in (qs, ks, vs, q_ropeds, outs)]
+    st = lib().sdvg_block_steps(n, cache.handle, *[C.cast(a, _VP) for a in arrays], grid[0], grid[1], grid[2],
+                                frame_offset, _ptr(table), tab_frames, block_index, scale, workspace.data_ptr(),
+                                workspace.numel(), _stream(stream))
+    _check(st, "sdvg_block_steps")
+
+
+def sdvg_block_steps_e4m3(cache: Cache, qs, ks, vs, q8_ropeds, outs, q_inv_scale, k_inv_scale, v_inv_scale,
+                          qk_descale, v_descale, grid, frame_offset: int, table, tab_frames: int, block_index: int,
+                          scale: float, workspace: torch.Tensor, stream=None) -> None:
+    """The same over an 8-bit ring (q8_ropeds receive E4M3 codes)."""
+    n = len(qs)
+    if not (len(ks) == len(vs) == len(q8_ropeds) == len(outs) == n):
+        raise ValueError("one q, k, v, q8_roped and out per step")
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    bf = lambda t: _bf16(t, shape)
+    u8 = lambda t: _u8(t, shape)
+    arrays = [_ptr_array(qs, bf), _ptr_array(ks, bf), _ptr_array(vs, bf), _ptr_array(q8_ropeds, u8), _ptr_array(outs, bf)]
+    sc = [_scales(t, cache.heads) for t in (q_inv_scale, k_inv_scale, v_inv_scale, qk_descale, v_descale)]
+    st = lib().sdvg_block_steps_e4m3(n, cache.handle, *[C.cast(a, _VP) for a in arrays], *sc, grid[0], grid[1], grid[2],
+                                     frame_offset, _ptr(table), tab_frames, block_index, scale, workspace.data_ptr(),
+                                     workspace.numel(), _stream(stream))
+    _check(st, "sdvg_block_steps_e4m3")

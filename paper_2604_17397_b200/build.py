@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libsdvg.so")
-SOURCES = ["sdvg_host.cu", "rope_commit.cu", "route.cu", "state.cu", "quant.cu", "attn_fwd.cu"]
+SOURCES = ["sdvg_host.cu", "rope_commit.cu", "route.cu", "state.cu", "quant.cu", "steps.cu", "attn_fwd.cu"]
 
 
 def nvcc_path() -> str:

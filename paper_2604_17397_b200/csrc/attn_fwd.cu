@@ -82,9 +82,13 @@ struct Deadline {
 // Slow path of the bounded wait: poll until the phase completes or the deadline passes.  Kept out
 // of line of the first attempt so that the timer read never sits on the fast path.  (A suspend-time
 // hint on the try_wait makes the waiting threads poll less often but wake later: measured slower.)
+#ifndef SDVG_WAIT_MODE
+#define SDVG_WAIT_MODE 0
+#endif
 __device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity, uint64_t deadline_ns,
                                            unsigned int* status) {
   uint32_t ok;
+#if SDVG_WAIT_MODE == 0
   asm volatile(
       "{\n\t"
       ".reg .pred p, q;\n\t"
@@ -101,6 +105,72 @@ __device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity
       : "=r"(ok)
       : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
       : "memory");
+#elif SDVG_WAIT_MODE == 1
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u64 t;\n\t"
+      "SDVG_WAIT:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %4;\n\t"
+      "@p bra SDVG_DONE;\n\t"
+      "mov.u64 t, %%globaltimer;\n\t"
+      "setp.lt.u64 q, t, %3;\n\t"
+      "@q bra SDVG_WAIT;\n\t"
+      "SDVG_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity), "l"(deadline_ns), "r"(20000)
+      : "memory");
+#elif SDVG_WAIT_MODE == 3
+  // non-suspending polls (test_wait), the timer read once per 64 of them
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u64 t;\n\t"
+      ".reg .u32 n;\n\t"
+      "mov.u32 n, 0;\n\t"
+      "SDVG_WAIT:\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra SDVG_DONE;\n\t"
+      "add.u32 n, n, 1;\n\t"
+      "and.b32 n, n, 63;\n\t"
+      "setp.ne.u32 q, n, 0;\n\t"
+      "@q bra SDVG_WAIT;\n\t"
+      "mov.u64 t, %%globaltimer;\n\t"
+      "setp.lt.u64 q, t, %3;\n\t"
+      "@q bra SDVG_WAIT;\n\t"
+      "SDVG_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
+      : "memory");
+#else
+  // the timer is read once per 256 polls
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, q;\n\t"
+      ".reg .u64 t;\n\t"
+      ".reg .u32 n;\n\t"
+      "mov.u32 n, 0;\n\t"
+      "SDVG_WAIT:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra SDVG_DONE;\n\t"
+      "add.u32 n, n, 1;\n\t"
+      "and.b32 n, n, 255;\n\t"
+      "setp.ne.u32 q, n, 0;\n\t"
+      "@q bra SDVG_WAIT;\n\t"
+      "mov.u64 t, %%globaltimer;\n\t"
+      "setp.lt.u64 q, t, %3;\n\t"
+      "@q bra SDVG_WAIT;\n\t"
+      "SDVG_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
+      : "memory");
+#endif
   if (!ok) atomicMax(status, (unsigned)SDVG_ERR_TIMEOUT);      // sticky: only a reset clears it
   return ok != 0;
 }

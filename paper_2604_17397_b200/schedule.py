@@ -77,6 +77,23 @@ class ModelState:
                                       self.tab_frames, block, api.SDVG_STAGE)
             api.sdvg_block_attn_fwd(q_roped, None, None, self.cache, block, out, None, self.scale, self.workspace)
 
+    def block_steps(self, qs, ks, vs, block: int, q_ropeds, outs) -> None:
+        """All denoise steps of `block` in ONE library call (per step: fused rope (+ quantise) + stage, attention)."""
+        if self.e4m3:
+            api.sdvg_block_steps_e4m3(self.cache, qs, ks, vs, q_ropeds, outs, self.q_inv_scale, self.k_inv_scale,
+                                      self.v_inv_scale, self.qk_descale, self.v_descale, self.grid, block * self.frames,
+                                      self.table, self.tab_frames, block, self.scale, self.workspace)
+        else:
+            api.sdvg_block_steps(self.cache, qs, ks, vs, q_ropeds, outs, self.grid, block * self.frames, self.table,
+                                 self.tab_frames, block, self.scale, self.workspace)
+
+    def check_status(self, where: str) -> None:
+        """Raise if an attention kernel of this model gave up on a bounded wait since the workspace was last reset
+        (the status word is sticky, so one check covers every launch since then); synchronises the stream."""
+        st = api.sdvg_block_attn_status(self.workspace)
+        if st != api.SDVG_OK:
+            raise api.SdvgError(st, where)
+
     def commit_final(self, k, v, block: int) -> int:
         """Rope the block's final K and write it with V into the ring (SDVG_FINAL); returns the evicted block."""
         if self.e4m3:
@@ -141,16 +158,19 @@ def run_schedule(num_blocks: int, steps: int, scores: torch.Tensor, tau: float,
     for i in range(num_blocks):
         b = first_block_index + i
         res.drafter_attn_calls += _denoise("drafter", drafter, b, steps, provider, on_attention)
-        _, k, v = provider("drafter", b, "clean", 0)
-        res.drafter_evicted.append(_commit_clean(drafter, b, k, v))
         api.sdvg_route(flat[i * frames:(i + 1) * frames], None, 1, frames, b, tau, accept_d[i:i + 1],
                        qmin_d[i:i + 1], None)
-        accepted = bool(accept_d[i].item())
+        accepted = bool(accept_d[i].item())               # the flow's one synchronisation point per block
+        # a kernel that gave up leaves undefined outputs: stop before anything derived from them enters a ring
+        drafter.check_status(f"drafter steps of block {b}")
+        _, k, v = provider("drafter", b, "clean", 0)
+        res.drafter_evicted.append(_commit_clean(drafter, b, k, v))
         if accepted:
             _, k, v = provider("target", b, "accepted", 0)
             res.target_source.append("accepted")
         else:
             res.target_attn_calls += _denoise("target", target, b, steps, provider, on_attention)
+            target.check_status(f"target steps of block {b}")
             _, k, v = provider("target", b, "clean", 0)
             res.target_source.append("regenerated")
         res.target_evicted.append(_commit_clean(target, b, k, v))
@@ -162,9 +182,9 @@ def run_schedule(num_blocks: int, steps: int, scores: torch.Tensor, tau: float,
 class BlockStepGraph:
     """The S denoising steps of ONE block captured into a CUDA graph (Sec. 4.1: 4 steps per block).
 
-    Every step is the fused rope + stage call followed by the attention call, reading q, k, v from
-    fixed input tensors (``self.q[s]``, ``self.k[s]``, ``self.v[s]``: fill them before ``replay``) and
-    writing ``self.out[s]``.  The ring state does not change inside the loop (SDVG_STAGE leaves it
+    The capture holds ONE library call (sdvg_block_steps: per step the fused rope + stage kernel followed
+    by the attention kernel), reading q, k, v from fixed input tensors (``self.q[s]``, ``self.k[s]``,
+    ``self.v[s]``: fill them before ``replay``) and writing ``self.out[s]``.  The ring state does not change inside the loop (SDVG_STAGE leaves it
     alone), so the captured launches stay valid until the block's final commit; a new block needs a
     new capture because its ring slot, frame offset and key segments differ.  One eager pass runs
     first: the library's one-time set-up (kernel attributes, device queries) must not happen during
@@ -186,9 +206,7 @@ class BlockStepGraph:
             self._run()
 
     def _run(self):
-        m, b = self.m, self.block
-        for s in range(self.steps):
-            m.stage_and_attend(self.q[s], self.k[s], self.v[s], b, self.q_roped[s], self.out[s])
+        self.m.block_steps(self.q, self.k, self.v, self.block, self.q_roped, self.out)
 
     def replay(self):
         self.graph.replay()
