@@ -410,6 +410,19 @@ int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_
                              int64_t block_index, const float* qk_descale, const float* v_descale, void* out,
                              float* lse, float scale, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * sdvg_block_attn_fwd_batched for 8-bit rings: up to 4 independent problems of one shape (e.g. the conditional
+ * and the unconditional pass that a guidance scale of 3.0 implies, Sec. 4.1 "Models"), each with its own ring
+ * and its own scale vectors, in one launch when their key segments agree (else one launch each, in stream
+ * order).  All arrays are HOST arrays of `batch` entries; k_self8 / v_self8 / lse may be NULL (not given for
+ * any problem) or hold NULL entries.  Results equal those of separate sdvg_block_attn_fwd_e4m3 calls, bit for bit.
+ */
+int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const void* const* k_self8,
+                                     const void* const* v_self8, const sdvg_cache* const* caches,
+                                     const int64_t* block_index, const float* const* qk_descale,
+                                     const float* const* v_descale, void* const* out, float* const* lse, float scale,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- the denoising steps of a block in one call ------------------------------- */
 /*
  * Sec. 4.1 "Models": each block takes 4 denoising steps; Sec. 3 "Inference flow": the drafter pays them for

@@ -69,6 +69,7 @@ SIGNATURES = {
     "sdvg_rope3d_qk_commit_e4m3": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
                                         C.POINTER(_I64), _VP]),
     "sdvg_block_attn_fwd_e4m3": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
+    "sdvg_block_attn_fwd_e4m3_batched": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_steps": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _F, _VP, _SZ, _VP]),
     "sdvg_block_steps_e4m3": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I,
                                    _I64, _F, _VP, _SZ, _VP]),
@@ -491,3 +492,28 @@ def sdvg_block_steps_e4m3(cache: Cache, qs, ks, vs, q8_ropeds, outs, q_inv_scale
                                      frame_offset, _ptr(table), tab_frames, block_index, scale, workspace.data_ptr(),
                                      workspace.numel(), _stream(stream))
     _check(st, "sdvg_block_steps_e4m3")
+
+
+def sdvg_block_attn_fwd_e4m3_batched(q8s, k_self8s, v_self8s, caches, block_indices, qk_descales, v_descales, outs, lses,
+                                     scale: float, workspace: torch.Tensor, stream=None) -> None:
+    """Lists of per-problem arguments over 8-bit rings (k_self8s / v_self8s / lses may be None)."""
+    n = len(q8s)
+    shape = (caches[0].block_tokens, caches[0].heads, caches[0].head_dim)
+    heads = caches[0].heads
+
+    def arr(ts, check):
+        return None if ts is None else (_VP * n)(*[check(t) for t in ts])
+
+    def lse_ptr(t):
+        if t is not None and (t.dtype != torch.float32 or tuple(t.shape) != (shape[1], shape[0])):
+            raise ValueError("lse must be float32 [heads, block_tokens]")
+        return _ptr(t)
+
+    u8 = lambda t: _u8(t, shape)
+    sc = lambda t: _scales(t, heads)
+    keep = [arr(q8s, u8), arr(k_self8s, u8), arr(v_self8s, u8), (_VP * n)(*[c.handle.value for c in caches]),
+            (_I64 * n)(*block_indices), arr(qk_descales, sc), arr(v_descales, sc), arr(outs, lambda t: _bf16(t, shape)),
+            arr(lses, lse_ptr)]
+    st = lib().sdvg_block_attn_fwd_e4m3_batched(n, *[C.cast(a, _VP) if a is not None else None for a in keep], scale,
+                                                workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "sdvg_block_attn_fwd_e4m3_batched")

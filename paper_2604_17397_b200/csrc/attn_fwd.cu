@@ -45,6 +45,8 @@ struct alignas(64) AttnProblem {
   CUtensorMap v_map[kMaxSegments];
   __nv_bfloat16* out;
   float* lse;
+  const float* qk_descale;             // 8-bit variant only: per head, q scale * k scale
+  const float* v_descale;              // 8-bit variant only: per head, v scale
 };
 
 // All problems of a launch have the same shape and the same key segments (same ring fill, same
@@ -57,8 +59,6 @@ struct alignas(64) AttnParams {
   int tokens, heads;
   float scale_log2e;                   // scale * log2(e): softmax is evaluated with exp2
   unsigned int* work;                  // [0] self-test result, [1] sticky status word, [2] count of accumulator rescale events
-  const float* qk_descale;             // 8-bit variant only: per head, q scale * k scale
-  const float* v_descale;              // 8-bit variant only: per head, v scale
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -80,15 +80,13 @@ struct Deadline {
 };
 
 // Slow path of the bounded wait: poll until the phase completes or the deadline passes.  Kept out
-// of line of the first attempt so that the timer read never sits on the fast path.  (A suspend-time
-// hint on the try_wait makes the waiting threads poll less often but wake later: measured slower.)
-#ifndef SDVG_WAIT_MODE
-#define SDVG_WAIT_MODE 0
-#endif
+// of line of the first attempt so that the timer read never sits on the fast path.  Waiting threads
+// that poll less often (a suspend-time hint on the try_wait, the timer read once per 256 polls) or that
+// never suspend (test_wait) were measured 2-5% slower: how soon a waiter notices counts for more than the
+// issue slots its polling takes.
 __device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity, uint64_t deadline_ns,
                                            unsigned int* status) {
   uint32_t ok;
-#if SDVG_WAIT_MODE == 0
   asm volatile(
       "{\n\t"
       ".reg .pred p, q;\n\t"
@@ -105,72 +103,6 @@ __device__ __forceinline__ bool wait_bar_slow(uint32_t bar_addr, uint32_t parity
       : "=r"(ok)
       : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
       : "memory");
-#elif SDVG_WAIT_MODE == 1
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, q;\n\t"
-      ".reg .u64 t;\n\t"
-      "SDVG_WAIT:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %4;\n\t"
-      "@p bra SDVG_DONE;\n\t"
-      "mov.u64 t, %%globaltimer;\n\t"
-      "setp.lt.u64 q, t, %3;\n\t"
-      "@q bra SDVG_WAIT;\n\t"
-      "SDVG_DONE:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t"
-      "}"
-      : "=r"(ok)
-      : "r"(bar_addr), "r"(parity), "l"(deadline_ns), "r"(20000)
-      : "memory");
-#elif SDVG_WAIT_MODE == 3
-  // non-suspending polls (test_wait), the timer read once per 64 of them
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, q;\n\t"
-      ".reg .u64 t;\n\t"
-      ".reg .u32 n;\n\t"
-      "mov.u32 n, 0;\n\t"
-      "SDVG_WAIT:\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra SDVG_DONE;\n\t"
-      "add.u32 n, n, 1;\n\t"
-      "and.b32 n, n, 63;\n\t"
-      "setp.ne.u32 q, n, 0;\n\t"
-      "@q bra SDVG_WAIT;\n\t"
-      "mov.u64 t, %%globaltimer;\n\t"
-      "setp.lt.u64 q, t, %3;\n\t"
-      "@q bra SDVG_WAIT;\n\t"
-      "SDVG_DONE:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t"
-      "}"
-      : "=r"(ok)
-      : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
-      : "memory");
-#else
-  // the timer is read once per 256 polls
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, q;\n\t"
-      ".reg .u64 t;\n\t"
-      ".reg .u32 n;\n\t"
-      "mov.u32 n, 0;\n\t"
-      "SDVG_WAIT:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra SDVG_DONE;\n\t"
-      "add.u32 n, n, 1;\n\t"
-      "and.b32 n, n, 255;\n\t"
-      "setp.ne.u32 q, n, 0;\n\t"
-      "@q bra SDVG_WAIT;\n\t"
-      "mov.u64 t, %%globaltimer;\n\t"
-      "setp.lt.u64 q, t, %3;\n\t"
-      "@q bra SDVG_WAIT;\n\t"
-      "SDVG_DONE:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t"
-      "}"
-      : "=r"(ok)
-      : "r"(bar_addr), "r"(parity), "l"(deadline_ns)
-      : "memory");
-#endif
   if (!ok) atomicMax(status, (unsigned)SDVG_ERR_TIMEOUT);      // sticky: only a reset clears it
   return ok != 0;
 }
@@ -322,9 +254,16 @@ int fill_problem(AttnProblem& pr, int* seg_len, int* nseg_out, const void* q, co
 int attn_forward_batch(int batch, const void* const* q, const void* const* k_self, const void* const* v_self,
                        const sdvg_cache* const* caches, const int64_t* block_index, void* const* out,
                        float* const* lse, float scale, void* workspace, size_t workspace_bytes, cudaStream_t stream,
-                       int elem_bytes = 2, const float* qk_descale = nullptr, const float* v_descale = nullptr) {
+                       int elem_bytes = 2, const float* const* qk_descale = nullptr,
+                       const float* const* v_descale = nullptr) {
   if (batch < 1 || !q || !caches || !block_index || !out || !workspace) return SDVG_ERR_INVALID_ARG;
-  if (elem_bytes == 1 && (batch != 1 || !qk_descale || !v_descale)) return SDVG_ERR_INVALID_ARG;
+  if (elem_bytes == 1) {
+    if (!qk_descale || !v_descale) return SDVG_ERR_INVALID_ARG;
+    for (int b = 0; b < batch && b < kMaxBatch; ++b) {
+      if (!qk_descale[b] || !v_descale[b]) return SDVG_ERR_INVALID_ARG;
+      if ((reinterpret_cast<uintptr_t>(qk_descale[b]) | reinterpret_cast<uintptr_t>(v_descale[b])) & 3) return SDVG_ERR_MISALIGNED;
+    }
+  }
   if (batch > kMaxBatch) return SDVG_ERR_BAD_SHAPE;
   if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
   if (!(scale > 0.f) || !isfinite(scale)) return SDVG_ERR_INVALID_ARG;
@@ -347,8 +286,6 @@ int attn_forward_batch(int batch, const void* const* q, const void* const* k_sel
   p.heads = caches[0]->heads;
   p.scale_log2e = scale * 1.4426950408889634f;
   p.work = (unsigned int*)workspace;
-  p.qk_descale = qk_descale;
-  p.v_descale = v_descale;
   const int D = caches[0]->head_dim;
   bool same = true;
   int seg_len[kMaxBatch][kMaxSegments] = {}, nseg[kMaxBatch] = {};
@@ -356,6 +293,8 @@ int attn_forward_batch(int batch, const void* const* q, const void* const* k_sel
     st = fill_problem(p.prob[b], seg_len[b], &nseg[b], q[b], k_self ? k_self[b] : nullptr, v_self ? v_self[b] : nullptr,
                       caches[b], block_index[b], out[b], lse ? lse[b] : nullptr);
     if (st != SDVG_OK) return st;
+    p.prob[b].qk_descale = elem_bytes == 1 ? qk_descale[b] : nullptr;
+    p.prob[b].v_descale = elem_bytes == 1 ? v_descale[b] : nullptr;
     same = same && nseg[b] == nseg[0];
     for (int s = 0; same && s < nseg[b]; ++s) same = seg_len[b][s] == seg_len[0][s];
   }
@@ -437,15 +376,25 @@ int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* con
 int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_self8, const sdvg_cache* c,
                              int64_t block_index, const float* qk_descale, const float* v_descale, void* out,
                              float* lse, float scale, void* workspace, size_t workspace_bytes, void* stream_) {
-  if (!c || !qk_descale || !v_descale) return SDVG_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(qk_descale) | reinterpret_cast<uintptr_t>(v_descale)) & 3) return SDVG_ERR_MISALIGNED;
+  if (!c) return SDVG_ERR_INVALID_ARG;
   const void* const qs[1] = {q8};
   const void* const ks[1] = {k_self8};
   const void* const vs[1] = {v_self8};
   void* const outs[1] = {out};
   float* const lses[1] = {lse};
+  const float* const qkd[1] = {qk_descale};
+  const float* const vd[1] = {v_descale};
   return attn_forward_batch(1, qs, k_self8 ? ks : nullptr, v_self8 ? vs : nullptr, &c, &block_index, outs, lses, scale,
-                            workspace, workspace_bytes, (cudaStream_t)stream_, 1, qk_descale, v_descale);
+                            workspace, workspace_bytes, (cudaStream_t)stream_, 1, qkd, vd);
+}
+
+int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const void* const* k_self8,
+                                     const void* const* v_self8, const sdvg_cache* const* caches,
+                                     const int64_t* block_index, const float* const* qk_descale,
+                                     const float* const* v_descale, void* const* out, float* const* lse, float scale,
+                                     void* workspace, size_t workspace_bytes, void* stream_) {
+  return attn_forward_batch(batch, q8, k_self8, v_self8, caches, block_index, out, lse, scale, workspace,
+                            workspace_bytes, (cudaStream_t)stream_, 1, qk_descale, v_descale);
 }
 
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,

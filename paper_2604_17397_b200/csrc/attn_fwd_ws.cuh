@@ -604,7 +604,7 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       const int my_tile = i == 0 ? it.tile[0] : it.tile[1];
       const int my_head = i == 0 ? it.head[0] : it.head[1];
       if constexpr (F8) {                                  // the logit scale carries the head's q and k scales
-        c2 = p.scale_log2e * __ldg(p.qk_descale + my_head);
+        c2 = p.scale_log2e * __ldg(p.prob[my_head / p.heads].qk_descale + my_head % p.heads);
         c2x2 = pack2(c2, c2);
       }
       float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2 (+ the window shift)
@@ -762,7 +762,7 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       const int grow = my_tile * kTileM + row;
       const AttnProblem& pr = p.prob[my_head / p.heads];
       const int head = my_head % p.heads;
-      const float inv = F8 ? __ldg(p.v_descale + head) / l_run : 1.f / l_run;     // 8-bit: V's scale of this head
+      const float inv = F8 ? __ldg(pr.v_descale + head) / l_run : 1.f / l_run;     // 8-bit: V's scale of this head
       w0 *= inv;
       w1 *= inv;
 #pragma unroll 1
