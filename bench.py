@@ -36,7 +36,7 @@ ROUTE_FRAMES = 12
 ROUTE_BIG_BLOCKS = 1 << 20       # a batch large enough for the router to be bandwidth-bound (50 MB of scores)
 # DRAM bytes (read + write) of ONE attention launch from an ncu capture of the kernel as it stands; the
 # summaries are kept with the other profiler summaries.  None: not captured since the kernel last changed.
-ATTN_DRAM_BYTES_PER_LAUNCH = {"14b": None, "1.3b": None}
+ATTN_DRAM_BYTES_PER_LAUNCH = {"14b": 0.776e9, "1.3b": 0.1067e9}
 CPU_SAMPLE_HEADS = 12           # heads of one step the CPU oracle is timed on (about 10-20 s of host work)
 TIMED_LAUNCHES = 20             # launches per separately timed kernel (median and minimum are reported)
 BURST_REGION_S = 1.0            # a timed region shorter than this has not reached the power-capped regime
