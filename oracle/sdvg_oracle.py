@@ -402,19 +402,29 @@ def route_ref(scores: np.ndarray, frame_offsets, num_blocks: int, frames_per_blo
     minimum is taken left to right with a strict '<', so ties (and +0/-0) keep
     the lowest index; any NaN frame makes q_min that NaN (lowest such index)
     and the block is rejected.  Returns (accept u8[B], q_min f32[B], argmin i32[B]).
+
+    Ragged input the paper does not speak of (Eq. (1) presumes F >= 1 frames): a block
+    without frames is rejected with q_min NaN and argmin -1, and so is a block whose
+    range runs backwards or leaves [frame_offsets[0], frame_offsets[B]] (the offsets are
+    meant to be non-decreasing; only the two ends of the array are trusted).  With a
+    fixed frame count such a block cannot occur and frames_per_block < 1 is an error.
     """
     s = np.asarray(scores, dtype=np.float32).reshape(-1)
     tau32 = np.float32(tau)
     accept = np.zeros(num_blocks, dtype=np.uint8)
     q_min = np.zeros(num_blocks, dtype=np.float32)
     argmin = np.zeros(num_blocks, dtype=np.int32)
+    if frame_offsets is None and frames_per_block < 1:
+        raise ValueError("a block needs at least one frame")
     for b in range(num_blocks):
         if frame_offsets is None:
             lo, hi = b * frames_per_block, (b + 1) * frames_per_block
         else:
             lo, hi = int(frame_offsets[b]), int(frame_offsets[b + 1])
-        if hi <= lo:
-            raise ValueError("a block needs at least one frame")
+            all_lo, all_hi = int(frame_offsets[0]), int(frame_offsets[num_blocks])
+            if not (all_lo <= lo <= hi <= all_hi) or hi == lo:
+                q_min[b], argmin[b], accept[b] = np.float32(np.nan), -1, 0
+                continue
         m, idx = s[lo], 0
         for i in range(lo + 1, hi):
             x = s[i]
@@ -459,6 +469,11 @@ def route_policy_ref(scores, frame_offsets, num_blocks: int, frames_per_block: i
             lo, hi = b * frames_per_block, (b + 1) * frames_per_block
         else:
             lo, hi = int(frame_offsets[b]), int(frame_offsets[b + 1])
+            all_lo, all_hi = int(frame_offsets[0]), int(frame_offsets[num_blocks])
+            if not (all_lo <= lo <= hi <= all_hi) or hi == lo:
+                # no frames, or a malformed range: same reading as route_ref (rejected whatever the signal, NaN, -1)
+                aggv[b], argmin[b], accept[b] = np.float32(np.nan), -1, 0
+                continue
         if hi <= lo:
             raise ValueError("a block needs at least one frame")
         if agg == AGG_MIN:

@@ -5,7 +5,7 @@ import torch
 
 from oracle import sdvg_oracle as O
 from paper_2604_17397_b200 import api, synth
-from gpu_utils import ATTN_MAX_ABS, ATTN_MEAN_ABS, ATTN_REL_RMS, attn_errors, to_bits, to_dev
+from gpu_utils import ATTN_MAX_ABS, ATTN_MEAN_ABS, ATTN_REL_RMS, Canaries, attn_errors, to_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -23,13 +23,15 @@ def run_sequence(sh, nblocks, seed, staged, q_scale=1.0, with_lse=True, rows_per
     ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
     ws = api.attn_workspace()
     rng = np.random.default_rng(seed)
+    guard = Canaries()                       # guard bytes around every output and around the rings
+    guard.watch_cache(cache)
     for b in range(nblocks):
         q = synth.block_tensor(sh, seed, b, 0, synth.Q, std=q_scale)
         k = synth.block_tensor(sh, seed, b, 0, synth.K)
         v = synth.block_tensor(sh, seed, b, 0, synth.V)
         dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
-        out = torch.full_like(dq, float("nan"))
-        lse = torch.full((sh.heads, sh.block_tokens), float("nan"), device="cuda") if with_lse else None
+        out = guard.like(dq, float("nan"))
+        lse = guard.new((sh.heads, sh.block_tokens), torch.float32, float("nan")) if with_lse else None
         if staged:
             api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_STAGE)
             api.sdvg_block_attn_fwd(dq, None, None, cache, b, out, lse, sh.scale, ws)
@@ -52,6 +54,7 @@ def run_sequence(sh, nblocks, seed, staged, q_scale=1.0, with_lse=True, rows_per
                     assert np.allclose(lse.cpu().numpy()[h, rows], lse_ref[0], rtol=0, atol=2e-3)
         api.sdvg_kv_commit(cache, dk, dv, b, api.SDVG_FINAL)
         ref.commit(b, k, v, O.FINAL)
+        guard.check()
     cache.close()
 
 

@@ -6,7 +6,7 @@ import torch
 
 from oracle import sdvg_oracle as O
 from paper_2604_17397_b200 import api, synth
-from gpu_utils import f32_dev, to_bits, to_dev
+from gpu_utils import Canaries, f32_dev, to_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -105,6 +105,8 @@ def run_sequence(sh, nblocks, seed, q_std=1.0, k_gain=None, rows_per_head=None, 
     ring = O.RingCacheRef(sh.slots, H, sh.block_tokens, sh.head_dim, dtype=np.uint8)
     ws = api.attn_workspace()
     rng = np.random.default_rng(seed)
+    guard = Canaries()                       # guard bytes around the outputs and around the 8-bit rings
+    guard.watch_cache(cache)
     k_gain = np.ones(H, dtype=np.float32) if k_gain is None else np.asarray(k_gain, dtype=np.float32)
     # static scales sized for ~4.5 standard deviations of each tensor; different per head
     sq = (4.5 * q_std / 448 * (1 + 0.1 * np.arange(H))).astype(np.float32)
@@ -118,12 +120,12 @@ def run_sequence(sh, nblocks, seed, q_std=1.0, k_gain=None, rows_per_head=None, 
             k = O.f32_to_bf16(O.bf16_to_f32(k) * k_gain.reshape(1, -1, 1))
         v = synth.block_tensor(sh, seed, b, 0, synth.V)
         q8, k8, v8 = O.quant_e4m3_ref(q, 1 / sq), O.quant_e4m3_ref(k, 1 / sk), O.quant_e4m3_ref(v, 1 / sv)
-        dq8 = torch.zeros(q8.shape, dtype=torch.uint8, device="cuda")
+        dq8 = guard.new(q8.shape, torch.uint8)
         api.sdvg_quant_e4m3(to_dev(q), f32_dev(1 / sq), dq8)
         assert np.array_equal(dq8.cpu().numpy(), q8)
         api.sdvg_kv_commit_e4m3(cache, to_dev(k), to_dev(v), f32_dev(1 / sk), f32_dev(1 / sv), b, api.SDVG_STAGE)
-        out = torch.full((sh.block_tokens, H, sh.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
-        lse = torch.full((H, sh.block_tokens), float("nan"), device="cuda")
+        out = guard.new((sh.block_tokens, H, sh.head_dim), torch.bfloat16, float("nan"))
+        lse = guard.new((H, sh.block_tokens), torch.float32, float("nan"))
         api.sdvg_block_attn_fwd_e4m3(dq8, None, None, cache, b, f32_dev(qkd), f32_dev(vd), out, lse, sh.scale, ws)
         assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
         outs = [out]
@@ -154,6 +156,7 @@ def run_sequence(sh, nblocks, seed, q_std=1.0, k_gain=None, rows_per_head=None, 
             assert np.allclose(lse.cpu().numpy()[h, rows], lse_ref[0], rtol=0, atol=2e-3)
         api.sdvg_kv_commit_e4m3(cache, to_dev(k), to_dev(v), f32_dev(1 / sk), f32_dev(1 / sv), b, api.SDVG_FINAL)
         ring.commit(b, k8, v8, O.FINAL)
+        guard.check()
     cache.close()
 
 

@@ -5,7 +5,7 @@ import torch
 
 from oracle import sdvg_oracle as O
 from paper_2604_17397_b200 import api, synth
-from gpu_utils import to_bits, to_dev
+from gpu_utils import Canaries, to_bits, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -29,12 +29,14 @@ def test_rope_bit_exact(sh):
     q = synth.block_tensor(sh, 31, 1, 0, synth.Q)
     k = synth.block_tensor(sh, 31, 1, 0, synth.K)
     dq, dk = to_dev(q), to_dev(k)
-    oq, ok = torch.zeros_like(dq), torch.zeros_like(dk)
+    guard = Canaries()
+    oq, ok = guard.like(dq), guard.like(dk)
     api.sdvg_rope3d_qk(dq, dk, oq, ok, grid, fo, dev_tab, tabf)
     want_q = O.rope_bitspec(q, grid, fo, ref_tab, tabf)
     want_k = O.rope_bitspec(k, grid, fo, ref_tab, tabf)
     assert np.array_equal(to_bits(oq), want_q)
     assert np.array_equal(to_bits(ok), want_k)
+    guard.check()
     assert np.array_equal(to_bits(dq), q)              # inputs untouched
     # in place, and k alone
     api.sdvg_rope3d_qk(dq, None, dq, None, grid, fo, dev_tab, tabf)
@@ -60,6 +62,8 @@ def test_rope_close_to_fp64_rotation_on_gpu_output():
 def test_commit_ring_trace_and_contents(sh):
     cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
     ref = O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    guard = Canaries()
+    guard.watch_cache(cache)
     nblocks = 2 * sh.slots + 1
     for b in range(nblocks):
         k = synth.block_tensor(sh, 33, b, 0, synth.K)
@@ -82,6 +86,7 @@ def test_commit_ring_trace_and_contents(sh):
     for s in range(sh.slots):
         gk, gv = cache.read_block(s)
         assert np.array_equal(to_bits(gk), ref.k[s]) and np.array_equal(to_bits(gv), ref.v[s])
+    guard.check()
     cache.reset()
     assert cache.state() == (0, [-1] * sh.slots, -1)
     cache.close()
@@ -94,11 +99,13 @@ def test_fused_rope_commit_equals_two_calls_and_oracle(sh):
     grid = (sh.frames, sh.grid_h, sh.grid_w)
     fused = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
     split = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
+    guard = Canaries()
+    guard.watch_cache(fused)
     for b in range(3):
         q, k, v = (synth.block_tensor(sh, 34, b, 0, t) for t in (synth.Q, synth.K, synth.V))
         dq, dk, dv = to_dev(q), to_dev(k), to_dev(v)
         fo = b * sh.frames
-        q1, k1 = torch.empty_like(dq), torch.empty_like(dk)
+        q1, k1 = guard.like(dq), guard.like(dk)
         api.sdvg_rope3d_qk_commit(fused, dq, dk, dv, q1, k1 if b == 1 else None, grid, fo, dev_tab, tabf, b,
                                   api.SDVG_STAGE)
         assert fused.state()[2] == b
@@ -117,4 +124,5 @@ def test_fused_rope_commit_equals_two_calls_and_oracle(sh):
             gk, gv = c.read_block(b % sh.slots)
             assert np.array_equal(to_bits(gk), want_k)
             assert np.array_equal(to_bits(gv), v)
+    guard.check()
     assert fused.state() == split.state()

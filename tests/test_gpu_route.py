@@ -6,6 +6,7 @@ import torch
 from oracle import sdvg_oracle as O
 from paper_2604_17397_b200 import api, synth
 from conftest import read_golden_rows
+from gpu_utils import Canaries
 
 pytestmark = pytest.mark.gpu
 
@@ -13,11 +14,12 @@ pytestmark = pytest.mark.gpu
 def run_route(scores, offsets, nb, fpb, first, tau, want_argmin=True):
     s = torch.from_numpy(np.ascontiguousarray(scores, dtype=np.float32).reshape(-1)).cuda()
     off = None if offsets is None else torch.from_numpy(np.asarray(offsets, dtype=np.int32)).cuda()
-    acc = torch.full((nb,), 7, dtype=torch.uint8, device="cuda")
-    qm = torch.full((nb,), 123.0, dtype=torch.float32, device="cuda")
-    am = torch.full((nb,), -7, dtype=torch.int32, device="cuda") if want_argmin else None
+    guard = Canaries()                       # guard bytes around the three outputs
+    acc = guard.new((nb,), torch.uint8, 7)
+    qm = guard.new((nb,), torch.float32, 123.0)
+    am = guard.new((nb,), torch.int32, -7) if want_argmin else None
     api.sdvg_route(s, off, nb, fpb, first, tau, acc, qm, am)
-    torch.cuda.synchronize()
+    guard.check()
     return acc.cpu().numpy(), qm.cpu().numpy(), None if am is None else am.cpu().numpy()
 
 
@@ -108,3 +110,34 @@ def test_bandwidth_sized_batch_fixed_frames():
     # spot-check against the oracle proper on a slice that spans several tiles
     ref = O.route_ref(s[:3000].reshape(-1), None, 3000, 12, 0, -0.7)
     assert np.array_equal(ga[:3000], ref[0]) and np.array_equal(gi[:3000], ref[2])
+
+
+def test_malformed_offsets_read_nothing_out_of_range():
+    # Offsets live on the device, so the kernel guards itself: a block whose range runs backwards or leaves
+    # [offsets[0], offsets[B]) counts as a block without frames; a block that merely sits outside its tile's
+    # range (offsets not sorted) is still read where it is.  Same answers as the oracle's reading.
+    for row in read_golden_rows("route_malformed_cases.txt"):
+        offsets, scores, tau, accept, qmin, argmin = row
+        offs = np.array([int(t) for t in offsets.split()], dtype=np.int32)
+        s = np.array([float(t) for t in scores.split()], dtype=np.float32)
+        nb = offs.size - 1
+        got = run_route(s, offs, nb, 0, 1, float(tau))
+        ref = O.route_ref(s, offs, nb, 0, 1, float(tau))
+        want_acc = np.array([int(t) for t in accept.split()], dtype=np.uint8)
+        want_arg = np.array([int(t) for t in argmin.split()], dtype=np.int32)
+        want_q = np.array([float(t) for t in qmin.split()], dtype=np.float32)
+        for have in (got, ref):
+            assert np.array_equal(have[0], want_acc) and np.array_equal(have[2], want_arg)
+            assert np.array_equal(np.isnan(have[1]), np.isnan(want_q))
+            assert np.array_equal(have[1][~np.isnan(want_q)], want_q[~np.isnan(want_q)])
+    # a long, shuffled offset array: many tiles, most blocks outside their tile's range
+    rng = np.random.default_rng(5)
+    nb, f = 3000, 7
+    s = synth.normal_scores(nb, f, -0.5, 0.6, 6).reshape(-1)
+    starts = rng.permutation(nb).astype(np.int32) * f
+    offs = np.concatenate([[0], starts[1:], [nb * f]]).astype(np.int32)      # ends fixed, interior shuffled
+    got = run_route(s, offs, nb, 0, 1, -0.7)
+    ref = O.route_ref(s, offs, nb, 0, 1, -0.7)
+    assert np.array_equal(got[0], ref[0]) and np.array_equal(got[2], ref[2])
+    assert np.array_equal(got[1].view(np.uint32)[~np.isnan(ref[1])], ref[1].view(np.uint32)[~np.isnan(ref[1])])
+    assert np.array_equal(np.isnan(got[1]), np.isnan(ref[1]))

@@ -355,7 +355,20 @@ def test_route_ragged_and_streaming_offsets():
     a3, _, _ = O.route_ref(flat, offs, 5, 0, 0, -5.0)
     assert a3.tolist() == [0, 1, 1, 1, 1]
     with pytest.raises(ValueError):
-        O.route_ref(flat, np.array([0, 0, 3], dtype=np.int32), 2, 0, 0, -0.7)
+        O.route_ref(flat, None, 2, 0, 0, -0.7)                 # a fixed frame count below one
+
+
+def test_route_malformed_ragged_input_hand_worked():
+    # blocks without frames, offsets that run backwards or leave [offsets[0], offsets[B]]: rejected, NaN, -1
+    for offsets, scores, tau, accept, qmin, argmin in read_golden_rows("route_malformed_cases.txt"):
+        offs = np.array([int(t) for t in offsets.split()], dtype=np.int32)
+        s = np.array([float(t) for t in scores.split()], dtype=np.float32)
+        a, q, i = O.route_ref(s, offs, offs.size - 1, 0, 1, float(tau))
+        want_q = np.array([float(t) for t in qmin.split()], dtype=np.float32)
+        assert a.tolist() == [int(t) for t in accept.split()]
+        assert i.tolist() == [int(t) for t in argmin.split()]
+        assert np.array_equal(np.isnan(q), np.isnan(want_q))
+        assert np.array_equal(q[~np.isnan(want_q)], want_q[~np.isnan(want_q)])
 
 
 def test_route_degenerate_policies_and_accept_rate_convention():
