@@ -495,6 +495,29 @@ def e4m3_figures(st, pk, device):
             "note": "operands E4M3 with one static scale per head, P rounded to E4M3"}
 
 
+def projection_baseline(st, hbm, device):
+    """The model's QKV projection as a LIBRARY GEMM (torch.matmul; not part of the library or of any timed step):
+    the measured cost the fused rope + stage prologue follows, for judging a fusion of the prologue into the
+    projection's epilogue."""
+    torch, sh = st.torch, st.sh
+    d = sh.heads * sh.head_dim
+    x = torch.randn(sh.block_tokens, d, device=device, dtype=torch.bfloat16)
+    w = [torch.randn(d, 3 * d, device=device, dtype=torch.bfloat16) * 0.02 for _ in range(3)]     # 3 weight sets: > L2 in all
+    y = torch.empty(sh.block_tokens, 3 * d, device=device, dtype=torch.bfloat16)
+    ms = time_launches(torch, [lambda wi=wi: torch.matmul(x, wi, out=y) for wi in w])
+    flops = 2.0 * sh.block_tokens * d * 3 * d
+    s = stats(ms, flops, 1e-9)
+    pro = hbm["rope_stage_6pass"]["ms_median"]
+    t = st.tensor_bytes()
+    return {"what": "torch.matmul bf16 [%d, %d] x [%d, %d]: a stated library baseline outside the product path" %
+                    (sh.block_tokens, d, d, 3 * d),
+            "ms_median": s["ms_median"], "ms_min": s["ms_min"], "tflops": s["rate_median"],
+            "prologue_ms": pro, "prologue_share_of_projection": pro / s["ms_median"],
+            "fusion_saves_at_most_ms": 3 * t / (hbm["peak_gbs"] * 1e6),
+            "note": "a fused epilogue removes the prologue's read of q, k, v (3 tensor passes); q', k' and v still have to be "
+                    "written, so the saving is bounded by 3 passes at the copy rate"}
+
+
 def plumbing_only(args):
     """No GPU work: every rank joins a gloo group, the ranks report their place, rank 0 prints one line.
     Lets the launch path of --gpus N be exercised on a machine without GPUs."""
@@ -552,10 +575,11 @@ def run_ours(args):
     assert api.sdvg_block_attn_status(st.ws) == api.SDVG_OK, "attention kernel reported a timeout"
 
     secondary = rank == 0 and not args.headline_only
-    hbm = fills = sweep7 = sweep9 = pair = e4m3 = None
+    hbm = fills = sweep7 = sweep9 = pair = e4m3 = proj = None
     if secondary:
         hbm = hbm_kernel_figures(st, pk, device)
         if args.workload != "tiny":
+            proj = projection_baseline(st, hbm, device)
             fills = fill_level_figures(st, device)
             sweep7 = sweep_figures(st, device, sh.slots)
             sweep9 = sweep_figures(st, device, 9)
@@ -634,6 +658,7 @@ def run_ours(args):
         "sweep_9_blocks_x_4_steps": sweep9,
         "attention_guidance_pair": pair,
         "attention_e4m3": e4m3,
+        "qkv_projection_baseline": proj,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))

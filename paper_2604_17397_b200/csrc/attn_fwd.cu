@@ -361,6 +361,7 @@ int sdvg_block_attn_workspace_reset(void* workspace, size_t workspace_bytes, voi
 int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
                         int64_t block_index, void* out, float* lse, float scale, void* workspace,
                         size_t workspace_bytes, void* stream_) {
+  SDVG_RANGE();
   return attn_forward(q, k_self, v_self, c, block_index, out, lse, scale, workspace, workspace_bytes,
                       (cudaStream_t)stream_);
 }
@@ -369,6 +370,7 @@ int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* con
                                 const void* const* v_self, const sdvg_cache* const* caches,
                                 const int64_t* block_index, void* const* out, float* const* lse, float scale,
                                 void* workspace, size_t workspace_bytes, void* stream_) {
+  SDVG_RANGE();
   return attn_forward_batch(batch, q, k_self, v_self, caches, block_index, out, lse, scale, workspace,
                             workspace_bytes, (cudaStream_t)stream_);
 }
@@ -376,6 +378,7 @@ int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* con
 int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_self8, const sdvg_cache* c,
                              int64_t block_index, const float* qk_descale, const float* v_descale, void* out,
                              float* lse, float scale, void* workspace, size_t workspace_bytes, void* stream_) {
+  SDVG_RANGE();
   if (!c) return SDVG_ERR_INVALID_ARG;
   const void* const qs[1] = {q8};
   const void* const ks[1] = {k_self8};
@@ -393,6 +396,7 @@ int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const voi
                                      const int64_t* block_index, const float* const* qk_descale,
                                      const float* const* v_descale, void* const* out, float* const* lse, float scale,
                                      void* workspace, size_t workspace_bytes, void* stream_) {
+  SDVG_RANGE();
   return attn_forward_batch(batch, q8, k_self8, v_self8, caches, block_index, out, lse, scale, workspace,
                             workspace_bytes, (cudaStream_t)stream_, 1, qk_descale, v_descale);
 }
@@ -400,6 +404,7 @@ int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const voi
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,
                                 int64_t block_index, void* out, float* lse, float scale,
                                 void** scratch_device_ptr, void* stream_) {
+  SDVG_RANGE();
   static std::mutex mu;
   static void* scratch_of_device[kMaxDevices] = {};
   // The built-in scratch has a fixed size; refuse rather than overrun if the kernel ever needs more.

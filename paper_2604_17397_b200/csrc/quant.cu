@@ -69,6 +69,7 @@ extern "C" {
 
 int sdvg_quant_e4m3(const void* x, const float* inv_scale, void* out, int tokens, int heads, int head_dim,
                     void* stream) {
+  SDVG_RANGE();
   if (!x || !inv_scale || !out) return SDVG_ERR_INVALID_ARG;
   if (tokens <= 0 || heads <= 0 || !sdvg::head_dim_ok(head_dim)) return SDVG_ERR_BAD_SHAPE;
   if (!sdvg::aligned16(x) || !sdvg::aligned16(out) || (reinterpret_cast<uintptr_t>(inv_scale) & 3))
@@ -86,6 +87,7 @@ int sdvg_quant_e4m3(const void* x, const float* inv_scale, void* out, int tokens
 int sdvg_kv_commit_e4m3(sdvg_cache* c, const void* k_roped, const void* v, const float* k_inv_scale,
                         const float* v_inv_scale, int64_t block_index, int flags, int64_t* evicted_block,
                         void* stream) {
+  SDVG_RANGE();
   if (!c || !k_roped || !v || !k_inv_scale || !v_inv_scale) return SDVG_ERR_INVALID_ARG;
   if (c->elem_bytes != 1) return SDVG_ERR_BAD_SHAPE;
   if (!sdvg::aligned16(k_roped) || !sdvg::aligned16(v) ||

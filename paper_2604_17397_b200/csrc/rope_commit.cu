@@ -186,6 +186,7 @@ extern "C" {
 int sdvg_rope3d_qk(const void* q, const void* k, void* q_out, void* k_out, int tokens, int heads,
                    int head_dim, int frames, int grid_h, int grid_w, int frame_offset,
                    const float* cos_sin_tab, int tab_frames, void* stream) {
+  SDVG_RANGE();
   if ((q == nullptr) != (q_out == nullptr) || (k == nullptr) != (k_out == nullptr)) return SDVG_ERR_INVALID_ARG;
   if (!q && !k) return SDVG_ERR_INVALID_ARG;
   if (tokens <= 0 || heads <= 0 || !sdvg::head_dim_ok(head_dim)) return SDVG_ERR_BAD_SHAPE;
@@ -204,6 +205,7 @@ int sdvg_rope3d_qk(const void* q, const void* k, void* q_out, void* k_out, int t
 
 int sdvg_kv_commit(sdvg_cache* c, const void* k_roped, const void* v, int64_t block_index, int flags,
                    int64_t* evicted_block, void* stream) {
+  SDVG_RANGE();
   if (!c || !k_roped || !v) return SDVG_ERR_INVALID_ARG;
   if (c->elem_bytes != 2) return SDVG_ERR_BAD_SHAPE;          // an 8-bit cache takes sdvg_kv_commit_e4m3
   if (!sdvg::aligned16(k_roped) || !sdvg::aligned16(v)) return SDVG_ERR_MISALIGNED;
@@ -229,6 +231,7 @@ int sdvg_rope3d_qk_commit(sdvg_cache* c, const void* q, const void* k, const voi
                           void* k_out, int frames, int grid_h, int grid_w, int frame_offset,
                           const float* cos_sin_tab, int tab_frames, int64_t block_index, int flags,
                           int64_t* evicted_block, void* stream) {
+  SDVG_RANGE();
   if (!c || !k || !v) return SDVG_ERR_INVALID_ARG;
   if (c->elem_bytes != 2) return SDVG_ERR_BAD_SHAPE;
   if ((q == nullptr) != (q_out == nullptr)) return SDVG_ERR_INVALID_ARG;
@@ -260,6 +263,7 @@ int sdvg_rope3d_qk_commit_e4m3(sdvg_cache* c, const void* q, const void* k, cons
                                const float* q_inv_scale, const float* k_inv_scale, const float* v_inv_scale,
                                int frames, int grid_h, int grid_w, int frame_offset, const float* cos_sin_tab,
                                int tab_frames, int64_t block_index, int flags, int64_t* evicted_block, void* stream) {
+  SDVG_RANGE();
   if (!c || !k || !v || !k_inv_scale || !v_inv_scale) return SDVG_ERR_INVALID_ARG;
   if (c->elem_bytes != 1) return SDVG_ERR_BAD_SHAPE;
   if ((q == nullptr) != (q8_out == nullptr) || (q && !q_inv_scale)) return SDVG_ERR_INVALID_ARG;
@@ -289,6 +293,7 @@ int sdvg_rope3d_qk_commit_e4m3(sdvg_cache* c, const void* q, const void* k, cons
 }
 
 int sdvg_cache_read_block(const sdvg_cache* c, int slot, void* k_out, void* v_out, void* stream) {
+  SDVG_RANGE();
   if (!c || (!k_out && !v_out)) return SDVG_ERR_INVALID_ARG;
   if (slot < 0 || slot >= c->slots) return SDVG_ERR_INVALID_ARG;
   if (!sdvg::aligned16(k_out) || !sdvg::aligned16(v_out)) return SDVG_ERR_MISALIGNED;

@@ -182,6 +182,7 @@ int route_checks(const float* scores, const int32_t* frame_offsets, int num_bloc
 extern "C" int sdvg_route(const float* scores, const int32_t* frame_offsets, int num_blocks,
                           int frames_per_block, int64_t first_block_index, float tau, uint8_t* accept,
                           float* q_min, int32_t* argmin, void* stream) {
+  SDVG_RANGE();
   int st = route_checks(scores, frame_offsets, num_blocks, frames_per_block, accept, q_min, argmin);
   if (st != SDVG_OK || num_blocks == 0) return st;
   if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
@@ -194,6 +195,7 @@ extern "C" int sdvg_route_policy(const float* scores, const int32_t* frame_offse
                                  int frames_per_block, int64_t first_block_index, int blocks_per_video, float tau,
                                  int agg, int signal, int force_first, const float* uniforms, float accept_prob,
                                  uint8_t* accept, float* aggregate_out, int32_t* argmin, void* stream) {
+  SDVG_RANGE();
   if ((agg != SDVG_AGG_MIN && agg != SDVG_AGG_MEAN) || (signal != SDVG_SIGNAL_REWARD && signal != SDVG_SIGNAL_RANDOM))
     return SDVG_ERR_INVALID_ARG;
   if (blocks_per_video < 0 || (blocks_per_video > 0 && first_block_index < 0)) return SDVG_ERR_INVALID_ARG;
@@ -211,6 +213,7 @@ extern "C" int sdvg_route_policy(const float* scores, const int32_t* frame_offse
 
 extern "C" int sdvg_accept_stats(const uint8_t* accept, int num_blocks, int64_t first_block_index,
                                  int blocks_per_video, unsigned long long* counts, void* stream_) {
+  SDVG_RANGE();
   if (num_blocks < 0) return SDVG_ERR_BAD_SHAPE;
   if (!counts || (num_blocks > 0 && !accept)) return SDVG_ERR_INVALID_ARG;
   if (blocks_per_video < 0 || (blocks_per_video > 0 && first_block_index < 0)) return SDVG_ERR_INVALID_ARG;

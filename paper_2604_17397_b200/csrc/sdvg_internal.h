@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include <vector>
@@ -19,6 +20,17 @@ struct sdvg_cache {
 };
 
 namespace sdvg {
+
+// NVTX range over the host side of an entry point (argument checks, tensor maps, launch): a timeline
+// tool then shows which library call enqueued which kernels.  Costs a function-pointer test when no
+// tool is attached.
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+  Range(const Range&) = delete;
+  Range& operator=(const Range&) = delete;
+};
+#define SDVG_RANGE() ::sdvg::Range sdvg_range_(__func__)
 
 // Records a CUDA error for sdvg_last_cuda_error() and maps it to a status.
 int cuda_status(cudaError_t e);

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(kThreads) state_copy_kernel(const __grid_const
 
 extern "C" int sdvg_state_copy(const void* const* src, void* const* dst, const size_t* bytes, int count,
                                void* stream) {
+  SDVG_RANGE();
   if (count < 0 || count > kMaxSegments) return SDVG_ERR_BAD_SHAPE;
   if (count == 0) return SDVG_OK;
   if (!src || !dst || !bytes) return SDVG_ERR_INVALID_ARG;

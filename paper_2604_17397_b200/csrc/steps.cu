@@ -36,6 +36,7 @@ int sdvg_block_steps(int steps, sdvg_cache* cache, const void* const* q, const v
                      const void* const* v, void* const* q_roped, void* const* out, int frames, int grid_h,
                      int grid_w, int frame_offset, const float* cos_sin_tab, int tab_frames, int64_t block_index,
                      float scale, void* workspace, size_t workspace_bytes, void* stream) {
+  SDVG_RANGE();
   int st = check_steps(steps, cache, q, k, v, q_roped, out, block_index, workspace, workspace_bytes, scale, 2);
   if (st != SDVG_OK) return st;
   for (int s = 0; s < steps; ++s) {
@@ -56,6 +57,7 @@ int sdvg_block_steps_e4m3(int steps, sdvg_cache* cache, const void* const* q, co
                           const float* qk_descale, const float* v_descale, int frames, int grid_h, int grid_w,
                           int frame_offset, const float* cos_sin_tab, int tab_frames, int64_t block_index, float scale,
                           void* workspace, size_t workspace_bytes, void* stream) {
+  SDVG_RANGE();
   int st = check_steps(steps, cache, q, k, v, q8_roped, out, block_index, workspace, workspace_bytes, scale, 1);
   if (st != SDVG_OK) return st;
   if (!q_inv_scale || !k_inv_scale || !v_inv_scale || !qk_descale || !v_descale) return SDVG_ERR_INVALID_ARG;
