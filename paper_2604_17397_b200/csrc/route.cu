@@ -127,6 +127,45 @@ __global__ void __launch_bounds__(kThreads) route_kernel(const __grid_constant__
   }
 }
 
+// Fixed frame count that is a multiple of four, scores 16-byte aligned: a block's frames are F / 4 aligned
+// 16-byte vectors, so each thread reads its own block straight from global memory (a warp's loads cover one
+// contiguous run, every sector fully used; the vectors of a block after the first hit the line the first one
+// fetched) and no staging or barrier is needed.  Same left-to-right scan as above.
+template <int VECS>      // F / 4 when known at compile time (0: run-time count)
+__global__ void __launch_bounds__(kThreads) route_vec_kernel(const __grid_constant__ RouteParams p) {
+  const int vecs = VECS ? VECS : p.frames_per_block / 4;
+  for (int b = blockIdx.x * kThreads + threadIdx.x; b < p.num_blocks; b += gridDim.x * kThreads) {
+    const float4* src = reinterpret_cast<const float4*>(p.scores) + (long long)b * vecs;
+    float m;
+    int idx = -1;
+    if (p.agg == SDVG_AGG_MEAN) {
+      float4 x = __ldcs(src);
+      m = __fadd_rn(__fadd_rn(__fadd_rn(x.x, x.y), x.z), x.w);
+#pragma unroll 4
+      for (int i = 1; i < vecs; ++i) {
+        x = __ldcs(src + i);
+        m = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(m, x.x), x.y), x.z), x.w);
+      }
+      m = __fdiv_rn(m, (float)(4 * vecs));
+    } else {
+      // all vectors are requested before the scan; a NaN stops the scan where the sequential definition stops
+      float4 x = __ldcs(src);
+      m = x.x;
+      idx = 0;
+      auto step = [&](float v, int i) {
+        if (m == m && (v != v || v < m)) { m = v; idx = i; }
+      };
+      step(x.y, 1); step(x.z, 2); step(x.w, 3);
+#pragma unroll 4
+      for (int i = 1; i < vecs; ++i) {
+        x = __ldcs(src + i);
+        step(x.x, 4 * i); step(x.y, 4 * i + 1); step(x.z, 4 * i + 2); step(x.w, 4 * i + 3);
+      }
+    }
+    decide(p, b, m, idx, true);
+  }
+}
+
 // accept-rate statistics: counts[0] += accepted, counts[1] += routable, first blocks left out of both
 __global__ void __launch_bounds__(kThreads) accept_stats_kernel(const uint8_t* __restrict__ accept, int num_blocks,
                                                                  long long first_block_index, int blocks_per_video,
@@ -159,6 +198,12 @@ int route_launch(const RouteParams& p, cudaStream_t stream) {
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int ntiles = (p.num_blocks + kThreads - 1) / kThreads;
+  if (!p.offsets && p.frames_per_block % 4 == 0 && (reinterpret_cast<uintptr_t>(p.scores) & 15) == 0) {
+    const int grid = ntiles < sms * 32 ? ntiles : sms * 32;      // one block of scores per thread up to 1.2 M blocks
+    if (p.frames_per_block == 12) route_vec_kernel<3><<<grid, kThreads, 0, stream>>>(p);
+    else route_vec_kernel<0><<<grid, kThreads, 0, stream>>>(p);
+    return sdvg::cuda_status(cudaGetLastError());
+  }
   const int grid = ntiles < sms * 4 ? ntiles : sms * 4;
   route_kernel<<<grid, kThreads, 0, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());

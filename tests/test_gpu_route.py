@@ -141,3 +141,30 @@ def test_malformed_offsets_read_nothing_out_of_range():
     assert np.array_equal(got[0], ref[0]) and np.array_equal(got[2], ref[2])
     assert np.array_equal(got[1].view(np.uint32)[~np.isnan(ref[1])], ref[1].view(np.uint32)[~np.isnan(ref[1])])
     assert np.array_equal(np.isnan(got[1]), np.isnan(ref[1]))
+
+
+@pytest.mark.parametrize("frames", [4, 8, 12, 16, 20])
+def test_vector_path_special_values_at_every_position(frames):
+    # fixed frame counts that are multiples of four take the 16-byte vector path: NaN, +-Inf, ties and signed zeros
+    # at every frame position must resolve exactly as the sequential left-to-right definition does
+    rng = np.random.default_rng(frames)
+    nb = 4 * frames * 6 + 37
+    s = synth.normal_scores(nb, frames, -0.5, 0.6, 30 + frames)
+    specials = [np.nan, np.inf, -np.inf, -0.0, 0.0, -0.7]
+    b = 1
+    for pos in range(frames):
+        for v in specials:
+            s[b, pos] = v
+            if pos + 1 < frames and v == v:
+                s[b, pos + 1] = v                      # a tie right behind it
+            b += 1
+    for tau in (-0.7, 0.0):
+        assert_same(run_route(s, None, nb, frames, 0, tau), O.route_ref(s.reshape(-1), None, nb, frames, 0, tau))
+    # the same scores shifted by one float: no longer 16-byte aligned, so the staged path runs; same answers
+    flat = np.concatenate([[0.0], s.reshape(-1)]).astype(np.float32)
+    d = torch.from_numpy(flat).cuda()[1:]
+    acc = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    qm = torch.empty(nb, dtype=torch.float32, device="cuda")
+    am = torch.empty(nb, dtype=torch.int32, device="cuda")
+    api.sdvg_route(d, None, nb, frames, 0, -0.7, acc, qm, am)
+    assert_same((acc.cpu().numpy(), qm.cpu().numpy(), am.cpu().numpy()), O.route_ref(s.reshape(-1), None, nb, frames, 0, -0.7))
