@@ -529,6 +529,17 @@ def projection_baseline(st, hbm, device):
                     "written, so the saving is bounded by 3 passes at the copy rate"}
 
 
+def run_was_burst(clocks, region_s: float) -> bool:
+    """Which measured GEMM rate the attention kernel is held against depends on the regime the run was in.  With
+    clock samples (at least 5): a run whose median SM clock stayed at its maximum has not been pulled down by the
+    power cap (burst figure), one that ran below it is compared with the sustained figure.  Without samples: a timed
+    region of under a second counts as burst.  Both fractions are printed either way."""
+    have_clock = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks.get("samples", 0) >= 5)
+    if have_clock:
+        return clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"]
+    return region_s < BURST_REGION_S
+
+
 def plumbing_only(args):
     """No GPU work: every rank joins a gloo group, the ranks report their place, rank 0 prints one line.
     Lets the launch path of --gpus N be exercised on a machine without GPUs."""
@@ -625,13 +636,8 @@ def run_ours(args):
     attn_tflops = flops / (attn_ms * 1e-3) / 1e12
     h2d, d2h = st.e2e_bytes()
     cpu = run_oracle(sh, steps=1, warmup=0, heads_sampled=CPU_SAMPLE_HEADS) if world == 1 and not args.no_cpu_baseline else None
-    # Which measured GEMM rate the attention kernel is held against depends on the regime this run was in.  With
-    # clock samples: a run whose median SM clock stayed at its maximum has not been pulled down by the power cap
-    # (burst figure), one that ran below it is compared with the sustained figure.  Without samples: a timed region
-    # of under a second counts as burst.  Both fractions are printed either way.
     region_s = ms_total * 1e-3
-    have_clock = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks.get("samples", 0) >= 5)
-    burst = clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"] if have_clock else region_s < BURST_REGION_S
+    burst = run_was_burst(clocks, region_s)
     peak = pk["bf16_tflops"] if burst else pk["bf16_tflops_sustained"]
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,

@@ -173,6 +173,13 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
   {
     std::lock_guard<std::mutex> lock(g_setup_mu);
     if (!sms_of_device[dev]) {
+      // The softmax warps grow their register count out of what the other warps of their sub-partition give
+      // back; a warp that asks for more than its sub-partition holds would wait forever.  The pool is what the
+      // kernel was compiled to launch with, so refuse to launch a build whose count does not cover the split.
+      cudaFuncAttributes attr;
+      e = cudaFuncGetAttributes(&attr, attn_fwd_ws_kernel<D, F8>);
+      if (e != cudaSuccess) return sdvg::cuda_status(e);
+      if (5 * attr.numRegs < 4 * WsCfg<D, F8>::kSoftmaxRegs + WsCfg<D, F8>::kIssueRegs) return SDVG_ERR_BAD_STATE;
       e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                WsCfg<D, F8>::kDynamic);
       if (e != cudaSuccess) return sdvg::cuda_status(e);
