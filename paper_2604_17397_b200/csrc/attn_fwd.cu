@@ -4,8 +4,8 @@
 //
 // Both products run on the 5th-generation tensor cores (tcgen05.mma, bf16 in, fp32 accumulators in
 // tensor memory).  Q, K and V tiles are staged in shared memory by TMA with the 128-byte swizzle;
-// S = Q K^T lands in TMEM, the softmax threads (one per query row) read it with tcgen05.ld, write
-// the bf16 probabilities back over the same TMEM columns, and O += P V takes P straight from TMEM
+// S = Q K^T lands in TMEM, the softmax threads (two per query row) read it with tcgen05.ld and write
+// the bf16 probabilities to TMEM columns of their own, and O += P V takes P straight from TMEM
 // and V from shared memory as an MN-major operand.  Keys arrive as up to three segments (runs of
 // ring slots and/or the block's own K/V tensors), each with its own tensor map whose row extent
 // ends at the segment so that TMA zero-fills the ragged last tile; those columns are masked to
@@ -15,8 +15,8 @@
 // scales; Sec. 2 names quantised attention as an orthogonal speed-up and fixes no format.
 //
 // Every wait on an mbarrier is bounded: kWaitLimitNs after kernel start a waiting thread gives up
-// and writes SDVG_ERR_TIMEOUT to the status word; all roles then fall through to the common exit,
-// which releases tensor memory.
+// and raises the (sticky) status word to SDVG_ERR_TIMEOUT; all roles then fall through to the common
+// exit, which releases tensor memory.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
