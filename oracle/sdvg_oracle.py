@@ -4,7 +4,8 @@ A plain, slow, fp64 NumPy statement of what the path computes: 3D-RoPE on q/k,
 block-causal attention of one block against the rolling KV cache, the ring
 commit with eviction, the worst-frame router with a forced rejection of block
 0, the per-block speculative schedule that strings them together, and the 8-bit
-(E4M3) variant of the cache and the attention.  Nothing
+(E4M3) variant of the cache and the attention, with one static scale per head or one
+power-of-two scale per tile of 128 tokens.  Nothing
 here is blocked, fused or tuned; library matmul/exp are used as single steps.
 
 Only tests, the smoke check and the bench's ``cpu_baseline`` leg may import
@@ -386,6 +387,80 @@ def block_attn_e4m3_ref(q8, k_self8, v_self8, cache: "RingCacheRef", block_index
     k_all = np.concatenate([kw, k_self8], axis=0)
     v_all = np.concatenate([vw, v_self8], axis=0)
     return attn_e4m3_ref(q8, k_all, v_all, qk_descale, v_descale, scale, heads=heads, rows=rows)
+
+
+# ---- finer scales: one power-of-two scale per tile of 128 consecutive tokens of a block and per head --------
+# (the library's choice again, Sec. 2 fixing none: the granularity at which a block's K/V enter the ring, so that
+# a block, or a stretch of one, with a different magnitude keeps the format's 3 mantissa bits)
+
+E4M3_TILE_TOKENS = 128
+E4M3_SCALE_EXP_MIN, E4M3_SCALE_EXP_MAX = -126, 120
+
+
+def e4m3_tile_scale_exponent(amax: float) -> int:
+    """The smallest integer e in [-126, 120] with amax <= 448 * 2^e: the tile's scale is 2^e, so that its
+    largest magnitude lands in (224, 448] whenever e is not clamped.  A non-finite amax takes the largest e."""
+    amax = float(amax)
+    if not np.isfinite(amax):
+        return E4M3_SCALE_EXP_MAX
+    for e in range(E4M3_SCALE_EXP_MIN, E4M3_SCALE_EXP_MAX + 1):
+        if amax <= 448.0 * 2.0 ** e:
+            return e
+    return E4M3_SCALE_EXP_MAX
+
+
+def quant_e4m3_tiled_ref(x_bits: np.ndarray):
+    """bf16 [tokens, heads, dim] -> (codes [tokens, heads, dim], scales float32 [heads, tiles]).
+    Tile t of head h is tokens [128 t, 128 t + 128) (the last one may be short); its scale is 2^e with e from
+    e4m3_tile_scale_exponent of the largest finite-or-infinite magnitude in the tile (NaN elements do not count);
+    codes are e4m3_encode(x / scale), the division by a power of two being exact."""
+    x = bf16_to_f64(x_bits)
+    T, H, D = x.shape
+    tiles = (T + E4M3_TILE_TOKENS - 1) // E4M3_TILE_TOKENS
+    codes = np.empty((T, H, D), dtype=np.uint8)
+    scales = np.empty((H, tiles), dtype=np.float32)
+    for h in range(H):
+        for t in range(tiles):
+            r0, r1 = t * E4M3_TILE_TOKENS, min(T, (t + 1) * E4M3_TILE_TOKENS)
+            tile = x[r0:r1, h, :]
+            mags = np.abs(tile[~np.isnan(tile)])
+            e = e4m3_tile_scale_exponent(mags.max() if mags.size else 0.0)
+            scales[h, t] = np.float32(2.0 ** e)
+            with np.errstate(over="ignore"):
+                codes[r0:r1, h, :] = e4m3_encode(tile * 2.0 ** -e)
+    return codes, scales
+
+
+def e4m3_token_scales(scales: np.ndarray, tokens: int) -> np.ndarray:
+    """Tile scales [heads, tiles] -> one scale per token [tokens, heads] (float64)."""
+    return np.repeat(np.asarray(scales, dtype=np.float64), E4M3_TILE_TOKENS, axis=1)[:, :tokens].T.copy()
+
+
+def attn_e4m3_rowscaled_ref(q8, q_scale, k8, k_scale, v8, v_scale, scale: float, heads=None, rows=None,
+                            row_chunk: int = 1024):
+    """Attention on operands dequantised with one scale per (token, head), in fp64, nothing else rounded:
+      q_i = q_scale[i, h] dec(q8_i), k_j = k_scale[j, h] dec(k8_j), v_j = v_scale[j, h] dec(v8_j),
+      o_i = sum_j softmax_j(scale <q_i, k_j>) v_j.
+    q_scale is [query tokens, heads], k_scale and v_scale [keys, heads].  Same return values as attn_ref."""
+    Tq, H, D = q8.shape
+    heads = list(range(H)) if heads is None else list(heads)
+    rows = np.arange(Tq) if rows is None else np.asarray(rows, dtype=np.int64)
+    q_scale, k_scale, v_scale = (np.asarray(a, dtype=np.float64) for a in (q_scale, k_scale, v_scale))
+    o = np.empty((rows.size, len(heads), D), dtype=np.float64)
+    lse = np.empty((len(heads), rows.size), dtype=np.float64)
+    for hi, h in enumerate(heads):
+        kh = e4m3_decode(k8[:, h, :]) * k_scale[:, h, None]
+        vh = e4m3_decode(v8[:, h, :]) * v_scale[:, h, None]
+        for r0 in range(0, rows.size, row_chunk):
+            rr = rows[r0:r0 + row_chunk]
+            qh = e4m3_decode(q8[rr, h, :]) * q_scale[rr, h, None]
+            s = (qh @ kh.T) * scale
+            m = s.max(axis=1, keepdims=True)
+            p = np.exp(s - m)
+            l = p.sum(axis=1, keepdims=True)
+            o[r0:r0 + rr.size, hi, :] = (p @ vh) / l
+            lse[hi, r0:r0 + rr.size] = (m + np.log(l))[:, 0]
+    return o, lse
 
 
 # --------------------------------------------------------------------------

@@ -102,3 +102,100 @@ def test_block_attention_e4m3_sees_the_same_window_as_the_bf16_ring():
     assert np.array_equal(o, o_direct)
     with pytest.raises(RuntimeError):
         O.block_attn_e4m3_ref(q8, blocks[5][0], blocks[5][1], ring, 4, ones, ones, 0.05)
+
+
+# ---- one power-of-two scale per tile of 128 tokens and head ------------------------------------------------
+
+
+def test_tile_scale_exponent_on_hand_values():
+    # 448 = 0.875 * 2^9 is the largest E4M3 value: amax = 448 fits scale 1, the next bf16 value (450) needs 2
+    cases = [(448.0, 0), (450.0, 1), (896.0, 1), (897.0, 2), (1.0, -8), (0.875, -9), (0.876, -8), (224.0, -1), (224.5, 0),
+             (3.0, -7), (2.0 ** -140, -126), (0.0, -126), (448.0 * 2.0 ** 120, 120), (3.3e38, 120), (np.inf, 120)]
+    for amax, e in cases:
+        assert O.e4m3_tile_scale_exponent(amax) == e, amax
+    # closed form away from the clamps: e = ceil(log2(amax / 448)), so amax / 2^e lies in (224, 448]
+    rng = np.random.default_rng(0)
+    for amax in np.exp(rng.uniform(-60, 60, 500)):
+        e = O.e4m3_tile_scale_exponent(amax)
+        assert 224.0 < amax / 2.0 ** e <= 448.0
+        assert e == int(np.ceil(np.log2(amax / 448.0)))
+
+
+def test_tiled_quantiser_against_torch_cast_and_tile_independence():
+    rng = np.random.default_rng(6)
+    T, H, D = 300, 3, 16                                  # three tiles, the last one of 44 tokens
+    gain = np.exp(rng.uniform(-6, 6, (3, H)))             # every (tile, head) at its own magnitude
+    x = rng.standard_normal((T, H, D)) * np.repeat(gain, 128, axis=0)[:T, :, None]
+    xb = O.f32_to_bf16(x.astype(np.float32))
+    codes, scales = O.quant_e4m3_tiled_ref(xb)
+    assert codes.shape == (T, H, D) and codes.dtype == np.uint8 and scales.shape == (H, 3) and scales.dtype == np.float32
+    xf = O.bf16_to_f64(xb)
+    for h in range(H):
+        for t in range(3):
+            tile = xf[128 * t:128 * t + 128, h]
+            sc = float(scales[h, t])
+            assert sc == 2.0 ** round(np.log2(sc))                                        # a power of two
+            assert 224.0 < np.abs(tile).max() / sc <= 448.0                               # the tile uses the top binade
+            want = torch.from_numpy(tile / sc).to(torch.float32).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+            assert np.array_equal(codes[128 * t:128 * t + 128, h], want)                  # torch's own cast of x / scale
+    # dequantised values are within 2^-4 of the input (3 mantissa bits), down to the tile's subnormal step
+    deq = O.e4m3_decode(codes) * O.e4m3_token_scales(scales, T)[:, :, None]
+    step = O.e4m3_token_scales(scales, T)[:, :, None] * 2.0 ** -10
+    assert np.all(np.abs(deq - xf) <= np.maximum(np.abs(xf) * 2.0 ** -4, step))
+    # changing one tile changes only that tile's codes and scale
+    xb2 = xb.copy()
+    xb2[130:140, 1] = O.f32_to_bf16(np.full((10, D), 1e4, dtype=np.float32))
+    codes2, scales2 = O.quant_e4m3_tiled_ref(xb2)
+    same = np.ones((T, H), dtype=bool)
+    same[128:256, 1] = False
+    assert np.array_equal(codes2[same], codes[same])
+    assert scales2[1, 1] == 32.0 and np.array_equal(np.delete(scales2.ravel(), 1 * 3 + 1), np.delete(scales.ravel(), 1 * 3 + 1))
+    # with one magnitude everywhere it is the static quantiser at the same scale
+    y = O.f32_to_bf16((rng.standard_normal((T, 1, D)) * 0.5).astype(np.float32))
+    y[::128, 0, 0] = O.f32_to_bf16(np.array([3.0], dtype=np.float32))[0]          # every tile's largest magnitude: 3 -> 2^-7
+    c3, s3 = O.quant_e4m3_tiled_ref(y)
+    assert np.all(s3 == np.float32(2.0 ** -7))
+    assert np.array_equal(c3, O.quant_e4m3_ref(y, np.array([2.0 ** 7], dtype=np.float32)))
+    # special values: a NaN element does not set the scale and becomes the NaN code; an all-zero tile takes the smallest scale
+    z = np.zeros((128, 1, D), dtype=np.uint16)
+    cz, sz = O.quant_e4m3_tiled_ref(z)
+    assert sz[0, 0] == np.float32(2.0 ** -126) and not cz.any()
+    z[3, 0, 2] = 0x7FC0                                      # NaN
+    z[5, 0, 1] = O.f32_to_bf16(np.array([1.0], dtype=np.float32))[0]
+    cz, sz = O.quant_e4m3_tiled_ref(z)
+    assert sz[0, 0] == np.float32(2.0 ** -8) and cz[3, 0, 2] == 0x7F and cz[5, 0, 1] == 0x78       # 256 = 1.0 * 2^8: code 0x78
+
+
+def test_rowscaled_attention_reduces_to_its_neighbours():
+    rng = np.random.default_rng(12)
+    T, L, H, D = 9, 300, 2, 16
+    q8 = rng.integers(0x28, 0x48, (T, H, D)).astype(np.uint8) | (rng.integers(0, 2, (T, H, D)) * 0x80).astype(np.uint8)
+    k8 = rng.integers(0x28, 0x48, (L, H, D)).astype(np.uint8) | (rng.integers(0, 2, (L, H, D)) * 0x80).astype(np.uint8)
+    v8 = rng.integers(0x10, 0x60, (L, H, D)).astype(np.uint8) | (rng.integers(0, 2, (L, H, D)) * 0x80).astype(np.uint8)
+    # (a) constant scales per head: the static-scale oracle
+    sq, sk, sv = np.array([0.5, 2.0]), np.array([0.25, 1.0]), np.array([4.0, 0.125])
+    o_a, lse_a = O.attn_e4m3_rowscaled_ref(q8, np.tile(sq, (T, 1)), k8, np.tile(sk, (L, 1)), v8, np.tile(sv, (L, 1)), 0.3)
+    o_b, lse_b = O.attn_e4m3_ref(q8, k8, v8, sq * sk, sv, 0.3)
+    np.testing.assert_allclose(o_a, o_b, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(lse_a, lse_b, rtol=1e-12, atol=1e-12)
+    # (b) power-of-two scales per tile: code * 2^e is a bf16 number, so the bf16 oracle on those numbers must agree
+    qs = O.e4m3_token_scales(2.0 ** rng.integers(-3, 3, (H, 1)), T)
+    ks = O.e4m3_token_scales(2.0 ** rng.integers(-3, 3, (H, 3)), L)
+    vs = O.e4m3_token_scales(2.0 ** rng.integers(-5, 5, (H, 3)), L)
+    o_c, lse_c = O.attn_e4m3_rowscaled_ref(q8, qs, k8, ks, v8, vs, 0.02)
+    deq = lambda c, s: O.f64_to_bf16(O.e4m3_decode(c) * s[:, :, None])
+    assert np.array_equal(O.bf16_to_f64(deq(k8, ks)), O.e4m3_decode(k8) * ks[:, :, None])          # exactly representable
+    o_d, lse_d = O.attn_ref(deq(q8, qs), deq(k8, ks), deq(v8, vs), 0.02)
+    np.testing.assert_allclose(o_c, o_d, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(lse_c, lse_d, rtol=1e-12, atol=1e-12)
+    # (c) heads and rows select; a key tile with a vanishing V scale contributes its weight but no value
+    o_e, _ = O.attn_e4m3_rowscaled_ref(q8, qs, k8, ks, v8, vs, 0.02, heads=[1], rows=[2, 7])
+    np.testing.assert_array_equal(o_e[:, 0], o_c[[2, 7], 1])
+    vs0 = vs.copy()
+    vs0[:128] = 0.0
+    o_f, lse_f = O.attn_e4m3_rowscaled_ref(q8, qs, k8, ks, v8, vs0, 0.02)
+    np.testing.assert_allclose(lse_f, lse_c, rtol=0, atol=0)
+    s = (O.e4m3_decode(q8[:, 0]) * qs[:, 0, None]) @ (O.e4m3_decode(k8[:, 0]) * ks[:, 0, None]).T * 0.02
+    p = np.exp(s - s.max(1, keepdims=True))
+    want = (p[:, 128:] @ (O.e4m3_decode(v8[128:, 0]) * vs[128:, 0, None])) / p.sum(1, keepdims=True)
+    np.testing.assert_allclose(o_f[:, 0], want, rtol=1e-12, atol=1e-12)
