@@ -423,6 +423,73 @@ int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const voi
                                      const float* const* v_descale, void* const* out, float* const* lse, float scale,
                                      void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- 8-bit variant with one scale per tile of 128 tokens ------------------------ */
+/*
+ * The same number format (Sec. 2 fixes none) with the scales chosen by the library from the data: every tile
+ * of 128 consecutive tokens of a block and every head has its own POWER-OF-TWO scale 2^e, e the smallest
+ * integer in [-126, 120] with max|x| <= 448 * 2^e over the tile (NaN elements do not count; an infinite
+ * maximum takes e = 120); codes are e4m3(x / 2^e), exact up to the one rounding of the conversion.  Nothing
+ * has to be calibrated, and a block, or a stretch of one, whose magnitude differs keeps the format's three
+ * mantissa bits.  tiles = ceil(block_tokens / 128); the last tile of a block may be short.
+ * An 8-bit ring takes such commits once its scale arrays are attached; the static-scale and the tile-scale
+ * entry points must not be mixed on one ring (the attention would read scales the other commit never wrote).
+ */
+
+/* Floats in ONE of the two scale arrays of a ring: heads * slots * tiles; 0 for a bad shape. */
+size_t sdvg_cache_tile_scale_floats(int slots, int heads, int block_tokens);
+
+/*
+ * Attaches the scale arrays of an 8-bit ring: device fp32 [heads][slots][tiles] each, caller-owned like the
+ * ring buffers and alive as long as the handle.  Errors: INVALID_ARG, BAD_SHAPE (bf16 ring), MISALIGNED
+ * (4 bytes).
+ */
+int sdvg_cache_set_tile_scales(sdvg_cache* cache, float* k_scale, float* v_scale);
+
+/*
+ * x: device bf16 [tokens, heads, 128] -> out8: device bytes, same shape, and tile_scale: device fp32
+ * [heads][tiles], as defined above.  Used for q when it is already rotated.
+ * Errors: INVALID_ARG, BAD_SHAPE (head_dim other than 128), MISALIGNED.
+ */
+int sdvg_quant_e4m3_tiled(const void* x, void* out8, float* tile_scale, int tokens, int heads, int head_dim,
+                          void* stream);
+
+/*
+ * sdvg_kv_commit for an 8-bit ring with tile scales: k_roped and v (device bf16 [block_tokens, heads, 128]) are
+ * quantised tile by tile into the slot, their scales into the attached arrays.  Same ordering rules, flags,
+ * eviction report and errors as sdvg_kv_commit; BAD_STATE also when no scale arrays are attached.
+ */
+int sdvg_kv_commit_e4m3_tiled(sdvg_cache* cache, const void* k_roped, const void* v, int64_t block_index,
+                              int flags, int64_t* evicted_block, void* stream);
+
+/*
+ * The fused prologue for such a ring, one pass: rope(q) -> q8_out with q_tile_scale [heads][tiles], rope(k) and
+ * v -> the ring slot of block_index with their scales.  rope() is the bit-specified rotation of sdvg_rope3d_qk
+ * including its rounding to bf16, so the result is bit-identical to sdvg_rope3d_qk followed by
+ * sdvg_quant_e4m3_tiled (q) and sdvg_kv_commit_e4m3_tiled (k, v).  q / q8_out / q_tile_scale may be NULL together.
+ * Other arguments and errors as sdvg_rope3d_qk_commit.
+ */
+int sdvg_rope3d_qk_commit_e4m3_tiled(sdvg_cache* cache, const void* q, const void* k, const void* v, void* q8_out,
+                                     float* q_tile_scale, int frames, int grid_h, int grid_w, int frame_offset,
+                                     const float* cos_sin_tab, int tab_frames, int64_t block_index, int flags,
+                                     int64_t* evicted_block, void* stream);
+
+/*
+ * sdvg_block_attn_fwd on such operands:
+ *   out[i, h, :] = sum_j softmax_j(scale * <sq_i dec q[i,h,:], sk_j dec K[j,h,:]>) sv_j dec V[j,h,:]
+ * with sq_i, sk_j, sv_j the scales of the tiles that query i and key j lie in, over the same visible keys.
+ * The block's own K/V must be staged in the ring (commit with SDVG_STAGE first); q8: device bytes
+ * [block_tokens, heads, 128]; q_tile_scale: device fp32 [heads][tiles]; out: device bf16; lse optional, as in
+ * sdvg_block_attn_fwd.  K's scale enters the logit scale of its key tile, V's scale the exponent of that
+ * tile's probabilities before they are rounded to E4M3 (relative to the largest V scale met so far in the row's
+ * pass over the keys; the accumulator is rescaled, exactly, when that rises), so the tensor-core work is that
+ * of sdvg_block_attn_fwd_e4m3.  Every ring slot is tiled on its own (the short last tile of a block is padded).
+ * Errors: those of sdvg_block_attn_fwd; BAD_SHAPE for a bf16 ring or more than 16 slots; BAD_STATE when the
+ * block is not staged or no scale arrays are attached.
+ */
+int sdvg_block_attn_fwd_e4m3_tiled(const void* q8, const float* q_tile_scale, const sdvg_cache* cache,
+                                   int64_t block_index, void* out, float* lse, float scale, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
 /* ---- the denoising steps of a block in one call ------------------------------- */
 /*
  * Sec. 4.1 "Models": each block takes 4 denoising steps; Sec. 3 "Inference flow": the drafter pays them for

@@ -69,6 +69,13 @@ SIGNATURES = {
     "sdvg_rope3d_qk_commit_e4m3": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
                                         C.POINTER(_I64), _VP]),
     "sdvg_block_attn_fwd_e4m3": (_I, [_VP, _VP, _VP, _VP, _I64, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
+    "sdvg_cache_tile_scale_floats": (_SZ, [_I, _I, _I]),
+    "sdvg_cache_set_tile_scales": (_I, [_VP, _VP, _VP]),
+    "sdvg_quant_e4m3_tiled": (_I, [_VP, _VP, _VP, _I, _I, _I, _VP]),
+    "sdvg_kv_commit_e4m3_tiled": (_I, [_VP, _VP, _VP, _I64, _I, C.POINTER(_I64), _VP]),
+    "sdvg_rope3d_qk_commit_e4m3_tiled": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
+                                              C.POINTER(_I64), _VP]),
+    "sdvg_block_attn_fwd_e4m3_tiled": (_I, [_VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_attn_fwd_e4m3_batched": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_steps": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _F, _VP, _SZ, _VP]),
     "sdvg_block_steps_e4m3": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I,
@@ -165,7 +172,8 @@ def sdvg_rope3d_qk(q, k, q_out, k_out, grid, frame_offset: int, table: torch.Ten
 class Cache:
     """Rolling KV cache: torch owns the two device buffers, the library the ring state."""
 
-    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int, device="cuda", e4m3: bool = False):
+    def __init__(self, slots: int, heads: int, block_tokens: int, head_dim: int, device="cuda", e4m3: bool = False,
+                 tile_scales: bool = False):
         sizer = lib().sdvg_cache_bytes_e4m3 if e4m3 else lib().sdvg_cache_bytes
         nbytes = sizer(slots, heads, block_tokens, head_dim)
         if nbytes == 0:
@@ -181,6 +189,15 @@ class Cache:
         create = lib().sdvg_cache_create_e4m3 if e4m3 else lib().sdvg_cache_create
         _check(create(C.byref(h), self.k_ptr, self.v_ptr, slots, heads, block_tokens, head_dim), "sdvg_cache_create")
         self.handle = h
+        # 8-bit ring with one scale per (head, slot, tile of 128 tokens): torch owns the two scale arrays as well
+        self.tile_scales = tile_scales
+        if tile_scales:
+            n = lib().sdvg_cache_tile_scale_floats(slots, heads, block_tokens)
+            self.tiles = n // (slots * heads)
+            self.k_scale = torch.ones((heads, slots, self.tiles), dtype=torch.float32, device=device)
+            self.v_scale = torch.ones((heads, slots, self.tiles), dtype=torch.float32, device=device)
+            _check(lib().sdvg_cache_set_tile_scales(h, self.k_scale.data_ptr(), self.v_scale.data_ptr()),
+                   "sdvg_cache_set_tile_scales")
 
     def close(self):
         if getattr(self, "handle", None) is not None and self.handle.value:
@@ -453,6 +470,55 @@ def sdvg_block_attn_fwd_e4m3(q8, k_self8, v_self8, cache: Cache, block_index: in
                                         _bf16(out, shape), _ptr(lse), scale, workspace.data_ptr(), workspace.numel(),
                                         _stream(stream))
     _check(st, "sdvg_block_attn_fwd_e4m3")
+
+
+def _tile_scales(t: Optional[torch.Tensor], heads: int, tokens: int):
+    if t is None:
+        return None
+    if t.dtype != torch.float32 or tuple(t.shape) != (heads, (tokens + 127) // 128) or not t.is_contiguous():
+        raise ValueError("tile scales must be contiguous float32 [heads, ceil(tokens / 128)]")
+    return _ptr(t)
+
+
+def sdvg_quant_e4m3_tiled(x, out8, tile_scale, stream=None) -> None:
+    tokens, heads, head_dim = x.shape
+    st = lib().sdvg_quant_e4m3_tiled(_bf16(x), _u8(out8, x.shape), _tile_scales(tile_scale, heads, tokens), tokens,
+                                     heads, head_dim, _stream(stream))
+    _check(st, "sdvg_quant_e4m3_tiled")
+
+
+def sdvg_kv_commit_e4m3_tiled(cache: Cache, k_roped, v, block_index: int, flags: int, stream=None) -> int:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    ev = _I64(-1)
+    st = lib().sdvg_kv_commit_e4m3_tiled(cache.handle, _bf16(k_roped, shape), _bf16(v, shape), block_index, flags,
+                                         C.byref(ev), _stream(stream))
+    _check(st, "sdvg_kv_commit_e4m3_tiled")
+    return ev.value
+
+
+def sdvg_rope3d_qk_commit_e4m3_tiled(cache: Cache, q, k, v, q8_out, q_tile_scale, grid, frame_offset: int, table,
+                                     tab_frames: int, block_index: int, flags: int, stream=None) -> int:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    frames, grid_h, grid_w = grid
+    ev = _I64(-1)
+    st = lib().sdvg_rope3d_qk_commit_e4m3_tiled(cache.handle, _bf16(q, None if q is None else shape), _bf16(k, shape),
+                                                _bf16(v, shape), _u8(q8_out, None if q8_out is None else shape),
+                                                _tile_scales(q_tile_scale, cache.heads, cache.block_tokens), frames,
+                                                grid_h, grid_w, frame_offset, _ptr(table), tab_frames, block_index,
+                                                flags, C.byref(ev), _stream(stream))
+    _check(st, "sdvg_rope3d_qk_commit_e4m3_tiled")
+    return ev.value
+
+
+def sdvg_block_attn_fwd_e4m3_tiled(q8, q_tile_scale, cache: Cache, block_index: int, out, lse, scale: float,
+                                   workspace: torch.Tensor, stream=None) -> None:
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    if lse is not None and (lse.dtype != torch.float32 or tuple(lse.shape) != (cache.heads, cache.block_tokens)):
+        raise ValueError("lse must be float32 [heads, block_tokens]")
+    st = lib().sdvg_block_attn_fwd_e4m3_tiled(_u8(q8, shape), _tile_scales(q_tile_scale, cache.heads, cache.block_tokens),
+                                              cache.handle, block_index, _bf16(out, shape), _ptr(lse), scale,
+                                              workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "sdvg_block_attn_fwd_e4m3_tiled")
 
 
 # ---------------------------------------------------------------- the steps of a block in one call

@@ -47,6 +47,10 @@ struct alignas(64) AttnProblem {
   float* lse;
   const float* qk_descale;             // 8-bit variant only: per head, q scale * k scale
   const float* v_descale;              // 8-bit variant only: per head, v scale
+  // 8-bit variant with tile scales only (k_map[0] and v_map[0] are then 4-D maps over the whole ring):
+  const float* q_tile_scale;           // [heads][query tiles]
+  const float* k_tile_scale;           // [heads][slots][tiles], the cache's arrays
+  const float* v_tile_scale;
 };
 
 // All problems of a launch have the same shape and the same key segments (same ring fill, same
@@ -59,7 +63,11 @@ struct alignas(64) AttnParams {
   int tokens, heads;
   float scale_log2e;                   // scale * log2(e): softmax is evaluated with exp2
   unsigned int* work;                  // [0] self-test result, [1] sticky status word, [2] count of accumulator rescale events
+  // tile scales: the keys are the tiles of ts_nslots ring slots, every slot tiled on its own (ts_tiles tiles)
+  int ts_nslots, ts_tiles, ts_cache_slots;
+  unsigned char ts_slot[16];
 };
+static_assert(sizeof(AttnParams) <= 4096, "kernel parameter space");
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -157,12 +165,27 @@ int make_map(CUtensorMap* m, const void* base, int head_dim, long long rows, int
   return r == CUDA_SUCCESS ? SDVG_OK : SDVG_ERR_CUDA;
 }
 
+// The whole byte ring [heads][slots][tokens][128] as (dim, token, slot, head): box = one 128-byte row x 128 tokens
+// of one slot and head; tokens past the block's end read as zero.
+int make_ring_map(CUtensorMap* m, const void* base, long long tokens, int slots, int heads) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return SDVG_ERR_CUDA;
+  cuuint64_t dims[4] = {128, (cuuint64_t)tokens, (cuuint64_t)slots, (cuuint64_t)heads};
+  cuuint64_t strides[3] = {128, (cuuint64_t)tokens * 128, (cuuint64_t)slots * tokens * 128};
+  cuuint32_t box[4] = {128, (cuuint32_t)kTileN, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SDVG_OK : SDVG_ERR_CUDA;
+}
+
 // One-time set-up per device and kernel instance: the opt-in to the kernel's dynamic shared memory is a
 // per-device attribute, and the grid is sized by that device's SM count.
 constexpr int kMaxDevices = 64;
 std::mutex g_setup_mu;
 
-template <int D, bool F8 = false>
+template <int D, bool F8 = false, bool TS = false>
 int launch_ws(const AttnParams& p, cudaStream_t stream) {
   static int sms_of_device[kMaxDevices] = {};          // 0: this device has not been set up yet
   int dev = 0;
@@ -177,10 +200,10 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
       // back; a warp that asks for more than its sub-partition holds would wait forever.  The pool is what the
       // kernel was compiled to launch with, so refuse to launch a build whose count does not cover the split.
       cudaFuncAttributes attr;
-      e = cudaFuncGetAttributes(&attr, attn_fwd_ws_kernel<D, F8>);
+      e = cudaFuncGetAttributes(&attr, attn_fwd_ws_kernel<D, F8, TS>);
       if (e != cudaSuccess) return sdvg::cuda_status(e);
       if (5 * attr.numRegs < 4 * WsCfg<D, F8>::kSoftmaxRegs + WsCfg<D, F8>::kIssueRegs) return SDVG_ERR_BAD_STATE;
-      e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      e = cudaFuncSetAttribute(attn_fwd_ws_kernel<D, F8, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                WsCfg<D, F8>::kDynamic);
       if (e != cudaSuccess) return sdvg::cuda_status(e);
       int n = 0;
@@ -192,7 +215,7 @@ int launch_ws(const AttnParams& p, cudaStream_t stream) {
   }
   const int total_tiles = ((p.tokens + kTileM - 1) / kTileM) * p.heads * p.batch;
   const int grid = total_tiles < sms ? total_tiles : sms;
-  attn_fwd_ws_kernel<D, F8><<<grid, WsCfg<D, F8>::kThreads, WsCfg<D, F8>::kDynamic, stream>>>(p);
+  attn_fwd_ws_kernel<D, F8, TS><<<grid, WsCfg<D, F8>::kThreads, WsCfg<D, F8>::kDynamic, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
 }
 
@@ -406,6 +429,51 @@ int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const voi
   SDVG_RANGE();
   return attn_forward_batch(batch, q8, k_self8, v_self8, caches, block_index, out, lse, scale, workspace,
                             workspace_bytes, (cudaStream_t)stream_, 1, qk_descale, v_descale);
+}
+
+int sdvg_block_attn_fwd_e4m3_tiled(const void* q8, const float* q_tile_scale, const sdvg_cache* c, int64_t block_index,
+                                   void* out, float* lse, float scale, void* workspace, size_t workspace_bytes,
+                                   void* stream_) {
+  SDVG_RANGE();
+  if (!q8 || !q_tile_scale || !c || !out || !workspace) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 1 || c->slots > 16) return SDVG_ERR_BAD_SHAPE;
+  if (!c->k_tile_scale || !c->v_tile_scale) return SDVG_ERR_BAD_STATE;
+  if (workspace_bytes < (size_t)kWorkspaceBytes) return SDVG_ERR_INVALID_ARG;
+  if (!(scale > 0.f) || !isfinite(scale)) return SDVG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return SDVG_ERR_MISALIGNED;
+  if (!sdvg::aligned16(q8) || !sdvg::aligned16(out) ||
+      ((reinterpret_cast<uintptr_t>(lse) | reinterpret_cast<uintptr_t>(q_tile_scale)) & 3))
+    return SDVG_ERR_MISALIGNED;
+  // the block's own K/V must sit staged in its slot: this variant reads keys from the ring only
+  if (block_index < 0 || block_index != c->next_block || c->staged_block != block_index) return SDVG_ERR_BAD_STATE;
+  const int T = c->block_tokens, H = c->heads, S = c->slots;
+  AttnParams p = {};
+  const int64_t first = block_index - (S - 1) > 0 ? block_index - (S - 1) : 0;
+  for (int64_t b = first; b <= block_index; ++b) {
+    const int s = (int)(b % S);
+    if (b < block_index && c->slot_block[s] != b) return SDVG_ERR_BAD_STATE;
+    p.ts_slot[p.ts_nslots++] = (unsigned char)s;
+  }
+  int st = sdvg::require_sm100();
+  if (st != SDVG_OK) return st;
+  p.batch = 1;
+  p.tokens = T;
+  p.heads = H;
+  p.scale_log2e = scale * 1.4426950408889634f;
+  p.work = (unsigned int*)workspace;
+  p.nseg = 1;                                       // one (4-D) map per tensor
+  p.ts_tiles = sdvg::scale_tiles(T);
+  p.ts_cache_slots = S;
+  AttnProblem& pr = p.prob[0];
+  pr.out = (__nv_bfloat16*)out;
+  pr.lse = lse;
+  pr.q_tile_scale = q_tile_scale;
+  pr.k_tile_scale = c->k_tile_scale;
+  pr.v_tile_scale = c->v_tile_scale;
+  if ((st = make_map(&pr.q_map, q8, 128, T, H, (size_t)H * 128, 128, 1)) != SDVG_OK) return st;
+  if ((st = make_ring_map(&pr.k_map[0], c->k_buf, T, S, H)) != SDVG_OK) return st;
+  if ((st = make_ring_map(&pr.v_map[0], c->v_buf, T, S, H)) != SDVG_OK) return st;
+  return launch_ws<128, true, true>(p, (cudaStream_t)stream_);
 }
 
 int sdvg_block_attn_fwd_noalloc(const void* q, const void* k_self, const void* v_self, const sdvg_cache* c,

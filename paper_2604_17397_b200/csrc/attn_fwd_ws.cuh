@@ -59,8 +59,8 @@ struct WsCfg {
   static constexpr int kKV = 2 * kTileBytes;
   static constexpr int kRowMax = kKV + kStages * kTileBytes;        // float [2 parities][2 lanes][2 halves][128]: partial row maxima
   static constexpr int kRowSum = kRowMax + 2 * 2 * 2 * 128 * 4;     // float [2 lanes][128]: the upper half's share of the row sum
-  static constexpr int kMerge = kRowSum + 2 * 128 * 4;              // float [2][128]: lane 1's -m*c2 and l when a split tile is merged
-  static constexpr int kBars = kMerge + 2 * 128 * 4;
+  static constexpr int kMerge = kRowSum + 2 * 128 * 4;              // float [2][128]: lane 1's -m*c2 and l when a split tile is merged, then its V scale exponent
+  static constexpr int kBars = kMerge + 2 * 128 * 4 + 16;
   static constexpr int kNumBars = 20 + 2 * kStages;
   static constexpr int kMisc = kBars + kNumBars * 8;                // tmem slot
   static constexpr int kTotal = kMisc + 16;
@@ -291,7 +291,9 @@ __device__ __forceinline__ void max_chunk(const uint32_t (&s)[32], float (&mx)[4
 }
 
 // Number of real keys in key tile `kt` of the concatenated key segments (the last tile of a segment may be ragged).
+template <bool TS>
 __device__ __forceinline__ int key_tile_valid(const AttnParams& p, int kt) {
+  if constexpr (TS) return min(kTileN, p.tokens - (kt % p.ts_tiles) * kTileN);      // every ring slot is tiled on its own
   int valid = kTileN;
   for (int seg = 0; seg < p.nseg; ++seg) {
     const int nt = (p.seg_len[seg] + kTileN - 1) / kTileN;
@@ -304,8 +306,9 @@ __device__ __forceinline__ int key_tile_valid(const AttnParams& p, int kt) {
   return valid;
 }
 
-template <int D, bool F8 = false>
+template <int D, bool F8 = false, bool TS = false>
 __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(const __grid_constant__ AttnParams p) {
+  static_assert(!TS || F8, "tile scales belong to the 8-bit variant");
   using C = WsCfg<D, F8>;
   using Mix = ExpMix<F8>;
   extern __shared__ uint8_t smem_raw[];
@@ -371,7 +374,9 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
   const Deadline dl{globaltimer_ns() + kWaitLimitNs, p.work + 1};
   const WsSchedule sched(p.tokens, p.heads * p.batch, gridDim.x);   // it.head[] are global heads: problem * heads + head
   int ntiles_k = 0;
-  for (int s = 0; s < p.nseg; ++s) ntiles_k += (p.seg_len[s] + kTileN - 1) / kTileN;
+  if constexpr (TS) ntiles_k = p.ts_nslots * p.ts_tiles;
+  else
+    for (int s = 0; s < p.nseg; ++s) ntiles_k += (p.seg_len[s] + kTileN - 1) / kTileN;
 
   if (warp >= C::kSoftmaxWarps) {
     // ================= producer / issuer warps: few registers ==================================
@@ -385,6 +390,20 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
 
       // one K or V tile of key tile j of `head` into the next ring stage
       auto load_kv = [&](bool is_v, int head, int j) {
+        if constexpr (TS) {
+          // one 4-D map over the whole byte ring (dim, token, slot, head): tile j of the visible slots, rows past
+          // the block's end read as zero
+          if (!(alive = wait_warp(&kv_empty[ring.stage], ring.phase ^ 1, dl))) return;
+          if (leader) {
+            mbar_expect_tx(&kv_full[ring.stage], C::kTileBytes);
+            const AttnProblem& pr = p.prob[0];
+            tma_load_4d(smem + C::kKV + ring.stage * C::kTileBytes, is_v ? &pr.v_map[0] : &pr.k_map[0],
+                        &kv_full[ring.stage], 0, (j % p.ts_tiles) * kTileN, p.ts_slot[j / p.ts_tiles], head);
+          }
+          ring.template advance<C::kStages>();
+          ++kv_issued;
+          return;
+        }
         int seg = 0, kt = j;
         for (; seg < p.nseg - 1; ++seg) {
           const int nt = (p.seg_len[seg] + kTileN - 1) / kTileN;
@@ -603,15 +622,26 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       const int my_nk = i == 0 ? it.nk[0] : it.nk[1];
       const int my_tile = i == 0 ? it.tile[0] : it.tile[1];
       const int my_head = i == 0 ? it.head[0] : it.head[1];
-      if constexpr (F8) {                                  // the logit scale carries the head's q and k scales
+      float c2_item = c2;                                  // tile scales: scale * log2(e) * this query tile's scale
+      if constexpr (TS) {
+        c2_item = p.scale_log2e * __ldg(p.prob[0].q_tile_scale + my_head * p.ts_tiles + my_tile);
+      } else if constexpr (F8) {                           // the logit scale carries the head's q and k scales
         c2 = p.scale_log2e * __ldg(p.prob[my_head / p.heads].qk_descale + my_head % p.heads);
         c2x2 = pack2(c2, c2);
       }
       float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2 (+ the window shift)
+      int lv_ref = 0;                                      // tile scales: exponent of the V scale that O is relative to
       #pragma unroll 1
       for (int j = 0; j < my_nk && alive; ++j) {          // this lane's j-th key tile
         // number of real keys in that tile: the last tile of a key segment may be ragged
-        const int valid = key_tile_valid(p, it.key_tile(i, j));
+        const int valid = key_tile_valid<TS>(p, it.key_tile(i, j));
+        float k_sc = 1.f, v_sc = 1.f;                      // tile scales: this key tile's K and V scales (powers of two),
+        if constexpr (TS) {                                // fetched ahead of the wait for the logits
+          const int kt = it.key_tile(i, j);
+          const int idx = (my_head * p.ts_cache_slots + p.ts_slot[kt / p.ts_tiles]) * p.ts_tiles + kt % p.ts_tiles;
+          k_sc = __ldg(p.prob[0].k_tile_scale + idx);
+          v_sc = __ldg(p.prob[0].v_tile_scale + idx);
+        }
         const uint32_t par = s_cnt & 1;
         if (!(alive = wait_bar(&s_full[i], par, dl))) break;
         tc_fence_after();
@@ -642,7 +672,39 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         // both threads of the row take the same decision from the same values
         float alpha = 1.f;
         bool moved = false;
-        if (j == 0) {
+        float neg_tile = 0.f, l_gain = 1.f;                // tile scales only
+        if constexpr (TS) {
+          // Logits of this tile are S * c2 with the tile's own K scale, so the reference maximum is kept in
+          // scaled units.  V's scale rides on P: P = 2^(x - m_ref + shift - d), d = lv_ref - lv >= 0, with lv_ref
+          // the largest V exponent met so far (O is rescaled, exactly, when it rises; the row sum never carries it).
+          // d stops at 64: beyond that the tile's values are below 2^-64 of what O holds and P may vanish, but
+          // the row sum still gets the tile's weights, scaled back by 2^d.
+          c2 = c2_item * k_sc;
+          c2x2 = pack2(c2, c2);
+          const int lv = (__float_as_int(v_sc) >> 23) - 127;
+          const float mx_s = mxa * c2;
+          if (j == 0) {
+            m_ref = mx_s;
+            lv_ref = lv;
+          } else {
+            if (mx_s - m_ref > RefMax<F8>::kLazy) {
+              alpha = fast_exp2(m_ref - mx_s);
+              l_run *= alpha;
+              m_ref = mx_s;
+              moved = true;
+            }
+            if (lv > lv_ref) {                             // the same for every row of the tile
+              const int up = lv - lv_ref;
+              alpha *= up > 126 ? 0.f : __int_as_float((127 - up) << 23);
+              lv_ref = lv;
+              moved = true;
+            }
+          }
+          neg = RefMax<F8>::kShift - m_ref;
+          const int d = min(lv_ref - lv, 64);
+          neg_tile = neg - (float)d;
+          l_gain = __int_as_float((127 + d) << 23);
+        } else if (j == 0) {
           m_ref = mxa;
           neg = __fmul_rn(-mxa, c2) + RefMax<F8>::kShift;
         } else if ((mxa - m_ref) * c2 > RefMax<F8>::kLazy) {
@@ -673,7 +735,7 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
           tc_fence_before();
         }
         // ---- P = 2^(c2 * (S - m_ref)) for this thread's 64 keys
-        const uint64_t negx2 = pack2(neg, neg);
+        const uint64_t negx2 = TS ? pack2(neg_tile, neg_tile) : pack2(neg, neg);
         uint64_t sum_a = pack2(0.f, 0.f), sum_b = sum_a;
         uint32_t pk0[F8 ? 8 : 16], pk1[F8 ? 8 : 16];
         if constexpr (F8) {
@@ -697,7 +759,8 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
           float a0, a1, b0, b1;
           unpack2(sum_a, a0, a1);
           unpack2(sum_b, b0, b1);
-          l_run += (a0 + a1) + (b0 + b1);
+          if constexpr (TS) l_run += ((a0 + a1) + (b0 + b1)) * l_gain;
+          else l_run += (a0 + a1) + (b0 + b1);
         }
         // the previous P of this lane must have been consumed: its product is commit number s_cnt - 1 on o_full
         if (s_cnt > 0) {
@@ -744,6 +807,7 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         if (i == 1) {
           s_merge[row] = neg;
           s_merge[128 + row] = l_run;
+          if (TS && row == 0) s_merge[256] = (float)lv_ref;
           tc_fence_before();
           mbar_arrive(lane1_done);
           alive = wait_bar(merge_done, spar, dl);
@@ -758,11 +822,20 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         w1 = fast_exp2(negm - neg1);
         l_run = l_run * w0 + l1 * w1;
         neg = negm;
+        if constexpr (TS) {                          // the two partial numerators are relative to their own V scales
+          const int lv1 = (int)s_merge[256];
+          const int top = max(lv_ref, lv1);
+          w0 *= lv_ref == top ? 1.f : (top - lv_ref > 126 ? 0.f : __int_as_float((127 - (top - lv_ref)) << 23));
+          w1 *= lv1 == top ? 1.f : (top - lv1 > 126 ? 0.f : __int_as_float((127 - (top - lv1)) << 23));
+          lv_ref = top;
+        }
       }
       const int grow = my_tile * kTileM + row;
       const AttnProblem& pr = p.prob[my_head / p.heads];
       const int head = my_head % p.heads;
-      const float inv = F8 ? __ldg(pr.v_descale + head) / l_run : 1.f / l_run;     // 8-bit: V's scale of this head
+      // 8-bit: V's scale of this head, or, with tile scales, the scale O ended up relative to
+      const float inv = TS ? __int_as_float((127 + lv_ref) << 23) / l_run
+                           : (F8 ? __ldg(pr.v_descale + head) / l_run : 1.f / l_run);
       w0 *= inv;
       w1 *= inv;
 #pragma unroll 1

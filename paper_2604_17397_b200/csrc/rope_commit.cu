@@ -132,6 +132,125 @@ __global__ void __launch_bounds__(kThreads) slot_read_kernel(const uint4* __rest
   }
 }
 
+// ---- 8-bit ring with one power-of-two scale per tile of 128 tokens and head ---------------------------------
+// A CTA owns one (tile, head) of one tensor: 128 rows of 256 bytes, 8 x 16 bytes per thread held in registers
+// between the two passes a data-dependent scale needs (largest magnitude, then quantise).  The rows are rotated
+// first where the tensor is q or k, rounded to bf16 exactly as the bf16 path rounds them.  HBM: 2 bytes read,
+// 1 written per element.
+struct TileQuantJob {
+  const uint4* src;             // bf16 [tokens, heads, 128]
+  uint2* dst;                   // codes; (token, head) row at dst + token * token_stride + head * head_stride (8-byte units)
+  long long token_stride, head_stride;
+  float* scale;                 // scale of (head, tile) at scale[head * scale_head_stride + tile]
+  long long scale_head_stride;
+  int rope;
+};
+
+struct TileQuantParams {
+  RopeCommitParams r;           // token count, head count and the rotary fields; its own jobs are unused
+  TileQuantJob job[kMaxJobs];
+};
+
+// The smallest e in [-126, 120] with amax <= 448 * 2^e (448 = 0.875 * 2^9); amax is >= 0 or +inf, never NaN.
+__device__ __forceinline__ int tile_scale_exponent(float amax) {
+  if (!(amax < __int_as_float(0x7f800000))) return 120;
+  if (amax == 0.f) return -126;
+  int x;
+  const float m = frexpf(amax, &x);               // amax = m * 2^x, m in [0.5, 1)
+  const int e = x - 9 + (m > 0.875f ? 1 : 0);
+  return e < -126 ? -126 : (e > 120 ? 120 : e);
+}
+
+__device__ __forceinline__ float abs_max2(float acc, uint32_t w) {
+  // fmaxf drops a NaN operand: NaN elements do not set the scale
+  return fmaxf(fmaxf(acc, fabsf(bf16_lo(w))), fabsf(bf16_hi(w)));
+}
+
+__global__ void __launch_bounds__(kThreads) tile_quant_kernel(const __grid_constant__ TileQuantParams p) {
+  constexpr int VPR = 16;                          // 16-byte vectors per (token, head) row of 128 bf16
+  constexpr int kRows = 128 / (kThreads / VPR);    // rows per thread: 8
+  const TileQuantJob job = p.job[blockIdx.z];
+  const int tile = blockIdx.x, h = blockIdx.y;
+  const int j = threadIdx.x & (VPR - 1), r0 = threadIdx.x / VPR;
+  __shared__ float s_max[kThreads / 32];
+  uint4 v[kRows];
+#pragma unroll
+  for (int i = 0; i < kRows; ++i) {
+    const int t = tile * 128 + r0 + i * (kThreads / VPR);
+    v[i] = t < p.r.tokens ? __ldcs(job.src + ((size_t)t * p.r.heads + h) * VPR + j) : make_uint4(0, 0, 0, 0);
+  }
+  if (job.rope) {
+    const int pairs_w = 64 - p.r.pairs_f - p.r.pairs_h;
+#pragma unroll
+    for (int i = 0; i < kRows; ++i) {
+      const int t = tile * 128 + r0 + i * (kThreads / VPR);
+      if (t >= p.r.tokens) continue;
+      const int f = t / p.r.grid_hw;
+      const int rem = t - f * p.r.grid_hw;
+      const int y = rem / p.r.grid_w;
+      const int x = rem - y * p.r.grid_w;
+      float2 cs[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int pr = 4 * j + e;
+        int idx;
+        if (pr < p.r.pairs_f) idx = (p.r.frame_offset + f) * p.r.pairs_f + pr;
+        else if (pr < p.r.pairs_f + p.r.pairs_h) idx = p.r.tab_h_off + y * p.r.pairs_h + (pr - p.r.pairs_f);
+        else idx = p.r.tab_w_off + x * pairs_w + (pr - p.r.pairs_f - p.r.pairs_h);
+        cs[e] = __ldg(p.r.tab + idx);
+      }
+      v[i].x = rotate_pair(v[i].x, cs[0]);
+      v[i].y = rotate_pair(v[i].y, cs[1]);
+      v[i].z = rotate_pair(v[i].z, cs[2]);
+      v[i].w = rotate_pair(v[i].w, cs[3]);
+    }
+  }
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < kRows; ++i) {
+    amax = abs_max2(amax, v[i].x);
+    amax = abs_max2(amax, v[i].y);
+    amax = abs_max2(amax, v[i].z);
+    amax = abs_max2(amax, v[i].w);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = s_max[0];
+#pragma unroll
+  for (int w = 1; w < kThreads / 32; ++w) amax = fmaxf(amax, s_max[w]);
+  const int e = tile_scale_exponent(amax);
+  const float inv = __int_as_float((127 - e) << 23);          // 2^-e, exact; -e is in [-120, 126]
+  if (threadIdx.x == 0) job.scale[(size_t)h * job.scale_head_stride + tile] = __int_as_float((127 + e) << 23);
+#pragma unroll
+  for (int i = 0; i < kRows; ++i) {
+    const int t = tile * 128 + r0 + i * (kThreads / VPR);
+    if (t < p.r.tokens)
+      job.dst[(size_t)t * job.token_stride + (size_t)h * job.head_stride + j] =
+          make_uint2(quant4(v[i].x, v[i].y, inv), quant4(v[i].z, v[i].w, inv));
+  }
+}
+
+int launch_tile_quant(const TileQuantParams& p, int njobs, cudaStream_t stream) {
+  const int tiles = sdvg::scale_tiles(p.r.tokens);
+  if (p.r.heads > 65535 || njobs > kMaxJobs) return SDVG_ERR_BAD_SHAPE;
+  tile_quant_kernel<<<dim3(tiles, p.r.heads, njobs), kThreads, 0, stream>>>(p);
+  return sdvg::cuda_status(cudaGetLastError());
+}
+
+// Ring jobs of a tile-scaled commit into `slot`: codes into the byte rings, scales into the cache's scale arrays.
+void tile_commit_jobs(TileQuantParams& p, int& n, const sdvg_cache* c, int slot, const void* k, const void* v, int rope_k) {
+  const int tiles = sdvg::scale_tiles(c->block_tokens);
+  const long long head_stride = (long long)c->slots * c->block_tokens * 16;      // 8-byte units per head of the ring
+  uint2* kslot = (uint2*)c->k_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  uint2* vslot = (uint2*)c->v_buf + sdvg::slot_offset(c, 0, slot) / 8;
+  p.job[n++] = TileQuantJob{(const uint4*)k, kslot, 16, head_stride, c->k_tile_scale + (size_t)slot * tiles,
+                            (long long)c->slots * tiles, rope_k};
+  p.job[n++] = TileQuantJob{(const uint4*)v, vslot, 16, head_stride, c->v_tile_scale + (size_t)slot * tiles,
+                            (long long)c->slots * tiles, 0};
+}
+
 struct RopeArgs {
   int frames, grid_h, grid_w, frame_offset, tab_frames;
   const float* tab;
@@ -288,6 +407,75 @@ int sdvg_rope3d_qk_commit_e4m3(sdvg_cache* c, const void* q, const void* k, cons
   p.job[p.njobs++] = TensorJob{(const uint4*)v, nullptr, nullptr, 0, nullptr, vslot, v_inv_scale};
   st = launch(p, c->head_dim, (cudaStream_t)stream, true);
   if (st != SDVG_OK) return st;
+  sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
+  return SDVG_OK;
+}
+
+int sdvg_quant_e4m3_tiled(const void* x, void* out8, float* tile_scale, int tokens, int heads, int head_dim,
+                          void* stream) {
+  SDVG_RANGE();
+  if (!x || !out8 || !tile_scale) return SDVG_ERR_INVALID_ARG;
+  if (tokens <= 0 || heads <= 0 || head_dim != 128) return SDVG_ERR_BAD_SHAPE;
+  if (!sdvg::aligned16(x) || !sdvg::aligned16(out8) || (reinterpret_cast<uintptr_t>(tile_scale) & 3))
+    return SDVG_ERR_MISALIGNED;
+  int st = sdvg::require_sm100();
+  if (st != SDVG_OK) return st;
+  TileQuantParams p = {};
+  p.r.tokens = tokens;
+  p.r.heads = heads;
+  p.job[0] = TileQuantJob{(const uint4*)x, (uint2*)out8, (long long)heads * 16, 16, tile_scale,
+                          sdvg::scale_tiles(tokens), 0};
+  return launch_tile_quant(p, 1, (cudaStream_t)stream);
+}
+
+int sdvg_kv_commit_e4m3_tiled(sdvg_cache* c, const void* k_roped, const void* v, int64_t block_index, int flags,
+                              int64_t* evicted_block, void* stream) {
+  SDVG_RANGE();
+  if (!c || !k_roped || !v) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 1) return SDVG_ERR_BAD_SHAPE;
+  if (!c->k_tile_scale || !c->v_tile_scale) return SDVG_ERR_BAD_STATE;
+  if (!sdvg::aligned16(k_roped) || !sdvg::aligned16(v)) return SDVG_ERR_MISALIGNED;
+  int slot = 0;
+  int st = sdvg::ring_begin_commit(c, block_index, flags, &slot);
+  if (st != SDVG_OK) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  TileQuantParams p = {};
+  p.r.tokens = c->block_tokens;
+  p.r.heads = c->heads;
+  int n = 0;
+  tile_commit_jobs(p, n, c, slot, k_roped, v, 0);
+  if ((st = launch_tile_quant(p, n, (cudaStream_t)stream)) != SDVG_OK) return st;
+  sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
+  return SDVG_OK;
+}
+
+int sdvg_rope3d_qk_commit_e4m3_tiled(sdvg_cache* c, const void* q, const void* k, const void* v, void* q8_out,
+                                     float* q_tile_scale, int frames, int grid_h, int grid_w, int frame_offset,
+                                     const float* cos_sin_tab, int tab_frames, int64_t block_index, int flags,
+                                     int64_t* evicted_block, void* stream) {
+  SDVG_RANGE();
+  if (!c || !k || !v) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 1) return SDVG_ERR_BAD_SHAPE;
+  if (!c->k_tile_scale || !c->v_tile_scale) return SDVG_ERR_BAD_STATE;
+  if ((q == nullptr) != (q8_out == nullptr) || (q && !q_tile_scale)) return SDVG_ERR_INVALID_ARG;
+  if (!sdvg::aligned16(q) || !sdvg::aligned16(k) || !sdvg::aligned16(v) || !sdvg::aligned16(q8_out) ||
+      (reinterpret_cast<uintptr_t>(q_tile_scale) & 3))
+    return SDVG_ERR_MISALIGNED;
+  TileQuantParams p = {};
+  p.r.tokens = c->block_tokens;
+  p.r.heads = c->heads;
+  int st = fill_rope(p.r, c->head_dim, c->block_tokens,
+                     RopeArgs{frames, grid_h, grid_w, frame_offset, tab_frames, cos_sin_tab});
+  if (st != SDVG_OK) return st;
+  int slot = 0;
+  if ((st = sdvg::ring_begin_commit(c, block_index, flags, &slot)) != SDVG_OK) return st;
+  if ((st = sdvg::require_sm100()) != SDVG_OK) return st;
+  int n = 0;
+  if (q)
+    p.job[n++] = TileQuantJob{(const uint4*)q, (uint2*)q8_out, (long long)c->heads * 16, 16, q_tile_scale,
+                              sdvg::scale_tiles(c->block_tokens), 1};
+  tile_commit_jobs(p, n, c, slot, k, v, 1);
+  if ((st = launch_tile_quant(p, n, (cudaStream_t)stream)) != SDVG_OK) return st;
   sdvg::ring_end_commit(c, block_index, flags, slot, evicted_block);
   return SDVG_OK;
 }

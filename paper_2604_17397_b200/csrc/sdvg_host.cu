@@ -158,6 +158,20 @@ int sdvg_cache_create_e4m3(sdvg_cache** out, void* k_buf, void* v_buf, int slots
   return st;
 }
 
+size_t sdvg_cache_tile_scale_floats(int slots, int heads, int block_tokens) {
+  if (slots <= 0 || heads <= 0 || block_tokens <= 0) return 0;
+  return (size_t)slots * heads * sdvg::scale_tiles(block_tokens);
+}
+
+int sdvg_cache_set_tile_scales(sdvg_cache* c, float* k_scale, float* v_scale) {
+  if (!c || !k_scale || !v_scale) return SDVG_ERR_INVALID_ARG;
+  if (c->elem_bytes != 1) return SDVG_ERR_BAD_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(k_scale) | reinterpret_cast<uintptr_t>(v_scale)) & 3) return SDVG_ERR_MISALIGNED;
+  c->k_tile_scale = k_scale;
+  c->v_tile_scale = v_scale;
+  return SDVG_OK;
+}
+
 int sdvg_cache_reset(sdvg_cache* c) {
   if (!c) return SDVG_ERR_INVALID_ARG;
   c->next_block = 0;

@@ -17,6 +17,10 @@ struct sdvg_cache {
   int64_t next_block;
   int64_t staged_block;                 // block whose provisional K/V sit in its slot, -1 if none
   std::vector<int64_t> slot_block;      // slot -> committed block, -1 = empty
+  // 8-bit ring with one power-of-two scale per (head, slot, tile of 128 tokens): device fp32 [heads][slots][tiles],
+  // caller-owned like the rings; null until sdvg_cache_set_tile_scales
+  float* k_tile_scale = nullptr;
+  float* v_tile_scale = nullptr;
 };
 
 namespace sdvg {
@@ -41,6 +45,9 @@ int require_sm100();
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline bool head_dim_ok(int d) { return d == 64 || d == 128; }
+
+constexpr int kScaleTileTokens = 128;   // tokens per scale tile of the tile-scaled 8-bit ring
+inline int scale_tiles(int block_tokens) { return (block_tokens + kScaleTileTokens - 1) / kScaleTileTokens; }
 
 // Element (not byte) offset of (head, slot, token 0, dim 0) in a cache buffer laid out [heads][slots][tokens][dim].
 inline size_t slot_offset(const sdvg_cache* c, int head, int slot) {
