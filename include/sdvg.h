@@ -523,6 +523,18 @@ int sdvg_block_steps_e4m3(int steps, sdvg_cache* cache, const void* const* q, co
                           const float* cos_sin_tab, int tab_frames, int64_t block_index, float scale,
                           void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * The same over a tile-scaled 8-bit ring: per step sdvg_rope3d_qk_commit_e4m3_tiled(..., q8_roped[s], q_tile_scale[s],
+ * ..., SDVG_STAGE) then sdvg_block_attn_fwd_e4m3_tiled(q8_roped[s], q_tile_scale[s], ...).  q_tile_scale: HOST array of
+ * `steps` device fp32 [heads][tiles] arrays.  Errors: those of the two calls, checked for all steps first where they
+ * do not depend on the device.
+ */
+int sdvg_block_steps_e4m3_tiled(int steps, sdvg_cache* cache, const void* const* q, const void* const* k,
+                                const void* const* v, void* const* q8_roped, float* const* q_tile_scale,
+                                void* const* out, int frames, int grid_h, int grid_w, int frame_offset,
+                                const float* cos_sin_tab, int tab_frames, int64_t block_index, float scale,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

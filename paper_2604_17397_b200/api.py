@@ -75,6 +75,8 @@ SIGNATURES = {
     "sdvg_kv_commit_e4m3_tiled": (_I, [_VP, _VP, _VP, _I64, _I, C.POINTER(_I64), _VP]),
     "sdvg_rope3d_qk_commit_e4m3_tiled": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _I,
                                               C.POINTER(_I64), _VP]),
+    "sdvg_block_steps_e4m3_tiled": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _F, _VP, _SZ,
+                                         _VP]),
     "sdvg_block_attn_fwd_e4m3_tiled": (_I, [_VP, _VP, _VP, _I64, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_attn_fwd_e4m3_batched": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _F, _VP, _SZ, _VP]),
     "sdvg_block_steps": (_I, [_I, _VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _VP, _I, _I64, _F, _VP, _SZ, _VP]),
@@ -558,6 +560,25 @@ def sdvg_block_steps_e4m3(cache: Cache, qs, ks, vs, q8_ropeds, outs, q_inv_scale
                                      frame_offset, _ptr(table), tab_frames, block_index, scale, workspace.data_ptr(),
                                      workspace.numel(), _stream(stream))
     _check(st, "sdvg_block_steps_e4m3")
+
+
+def sdvg_block_steps_e4m3_tiled(cache: Cache, qs, ks, vs, q8_ropeds, q_tile_scales, outs, grid, frame_offset: int, table,
+                                tab_frames: int, block_index: int, scale: float, workspace: torch.Tensor,
+                                stream=None) -> None:
+    """The same over a tile-scaled 8-bit ring (q8_ropeds receive E4M3 codes, q_tile_scales their scales)."""
+    n = len(qs)
+    if not (len(ks) == len(vs) == len(q8_ropeds) == len(q_tile_scales) == len(outs) == n):
+        raise ValueError("one q, k, v, q8_roped, q_tile_scale and out per step")
+    shape = (cache.block_tokens, cache.heads, cache.head_dim)
+    bf = lambda t: _bf16(t, shape)
+    u8 = lambda t: _u8(t, shape)
+    ts = lambda t: _tile_scales(t, cache.heads, cache.block_tokens)
+    arrays = [_ptr_array(qs, bf), _ptr_array(ks, bf), _ptr_array(vs, bf), _ptr_array(q8_ropeds, u8),
+              _ptr_array(q_tile_scales, ts), _ptr_array(outs, bf)]
+    st = lib().sdvg_block_steps_e4m3_tiled(n, cache.handle, *[C.cast(a, _VP) for a in arrays], grid[0], grid[1], grid[2],
+                                           frame_offset, _ptr(table), tab_frames, block_index, scale,
+                                           workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "sdvg_block_steps_e4m3_tiled")
 
 
 def sdvg_block_attn_fwd_e4m3_batched(q8s, k_self8s, v_self8s, caches, block_indices, qk_descales, v_descales, outs, lses,

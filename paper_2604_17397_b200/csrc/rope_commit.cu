@@ -161,35 +161,42 @@ __device__ __forceinline__ int tile_scale_exponent(float amax) {
   return e < -126 ? -126 : (e > 120 ? 120 : e);
 }
 
-__device__ __forceinline__ float abs_max2(float acc, uint32_t w) {
-  // fmaxf drops a NaN operand: NaN elements do not set the scale
-  return fmaxf(fmaxf(acc, fabsf(bf16_lo(w))), fabsf(bf16_hi(w)));
+// running maximum of |x| over bf16 pairs, two at a time; the maximum drops a NaN operand, so NaN elements do not set
+// the scale (an accumulator that starts at zero never becomes NaN)
+__device__ __forceinline__ uint32_t abs_max2(uint32_t acc, uint32_t w) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(acc), "r"(w & 0x7fff7fffu));
+  return r;
 }
 
-__global__ void __launch_bounds__(kThreads) tile_quant_kernel(const __grid_constant__ TileQuantParams p) {
+constexpr int kTileHeads = 4;      // heads a CTA walks with the same 128 tokens (their rotary factors stay in registers)
+constexpr int kTileThreads = 512;
+
+// ROPE: some job of the launch rotates (q, k); the thread then keeps the (cos, sin) pairs of its rows in registers
+// for all heads it walks, and two CTAs per SM overlap each other's loads; without them the registers go to the
+// next head's vectors, requested before the current head is reduced and stored.
+template <bool ROPE>
+__global__ void __launch_bounds__(kTileThreads, 2) tile_quant_kernel(const __grid_constant__ TileQuantParams p) {
   constexpr int VPR = 16;                          // 16-byte vectors per (token, head) row of 128 bf16
-  constexpr int kRows = 128 / (kThreads / VPR);    // rows per thread: 8
+  constexpr int kRowStep = kTileThreads / VPR;     // 32 rows per pass
+  constexpr int kRows = 128 / kRowStep;            // rows per thread: 4
+  constexpr int kWarps = kTileThreads / 32;
   const TileQuantJob job = p.job[blockIdx.z];
-  const int tile = blockIdx.x, h = blockIdx.y;
+  const int tile = blockIdx.x, h0 = blockIdx.y * kTileHeads;
+  const int nh = min(kTileHeads, p.r.heads - h0);
   const int j = threadIdx.x & (VPR - 1), r0 = threadIdx.x / VPR;
-  __shared__ float s_max[kThreads / 32];
-  uint4 v[kRows];
-#pragma unroll
-  for (int i = 0; i < kRows; ++i) {
-    const int t = tile * 128 + r0 + i * (kThreads / VPR);
-    v[i] = t < p.r.tokens ? __ldcs(job.src + ((size_t)t * p.r.heads + h) * VPR + j) : make_uint4(0, 0, 0, 0);
-  }
-  if (job.rope) {
+  const int t0 = tile * 128 + r0;                  // this thread's rows are t0 + i * kRowStep
+  __shared__ float s_max[2][kWarps];
+  float2 cs[ROPE ? kRows : 1][4];
+  if (ROPE && job.rope) {
     const int pairs_w = 64 - p.r.pairs_f - p.r.pairs_h;
 #pragma unroll
     for (int i = 0; i < kRows; ++i) {
-      const int t = tile * 128 + r0 + i * (kThreads / VPR);
-      if (t >= p.r.tokens) continue;
+      const int t = min(t0 + i * kRowStep, p.r.tokens - 1);
       const int f = t / p.r.grid_hw;
       const int rem = t - f * p.r.grid_hw;
       const int y = rem / p.r.grid_w;
       const int x = rem - y * p.r.grid_w;
-      float2 cs[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int pr = 4 * j + e;
@@ -197,45 +204,75 @@ __global__ void __launch_bounds__(kThreads) tile_quant_kernel(const __grid_const
         if (pr < p.r.pairs_f) idx = (p.r.frame_offset + f) * p.r.pairs_f + pr;
         else if (pr < p.r.pairs_f + p.r.pairs_h) idx = p.r.tab_h_off + y * p.r.pairs_h + (pr - p.r.pairs_f);
         else idx = p.r.tab_w_off + x * pairs_w + (pr - p.r.pairs_f - p.r.pairs_h);
-        cs[e] = __ldg(p.r.tab + idx);
+        cs[i][e] = __ldg(p.r.tab + idx);
       }
-      v[i].x = rotate_pair(v[i].x, cs[0]);
-      v[i].y = rotate_pair(v[i].y, cs[1]);
-      v[i].z = rotate_pair(v[i].z, cs[2]);
-      v[i].w = rotate_pair(v[i].w, cs[3]);
     }
   }
-  float amax = 0.f;
+  auto load = [&](uint4 (&v)[kRows], int h) {
 #pragma unroll
-  for (int i = 0; i < kRows; ++i) {
-    amax = abs_max2(amax, v[i].x);
-    amax = abs_max2(amax, v[i].y);
-    amax = abs_max2(amax, v[i].z);
-    amax = abs_max2(amax, v[i].w);
-  }
+    for (int i = 0; i < kRows; ++i) {
+      const int t = t0 + i * kRowStep;
+      v[i] = t < p.r.tokens ? __ldcs(job.src + ((size_t)t * p.r.heads + h) * VPR + j) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  uint4 v[kRows], nxt[ROPE ? 1 : kRows];
+  if (!ROPE) load(v, h0);
+#pragma unroll 1
+  for (int g = 0; g < nh; ++g) {
+    const int h = h0 + g;
+    if constexpr (ROPE) load(v, h);
+    else if (g + 1 < nh) load(nxt, h + 1);
+    if (ROPE && job.rope) {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
-  __syncthreads();
-  amax = s_max[0];
+      for (int i = 0; i < kRows; ++i) {
+        v[i].x = rotate_pair(v[i].x, cs[i][0]);
+        v[i].y = rotate_pair(v[i].y, cs[i][1]);
+        v[i].z = rotate_pair(v[i].z, cs[i][2]);
+        v[i].w = rotate_pair(v[i].w, cs[i][3]);
+      }
+    }
+    uint32_t am2 = 0;
 #pragma unroll
-  for (int w = 1; w < kThreads / 32; ++w) amax = fmaxf(amax, s_max[w]);
-  const int e = tile_scale_exponent(amax);
-  const float inv = __int_as_float((127 - e) << 23);          // 2^-e, exact; -e is in [-120, 126]
-  if (threadIdx.x == 0) job.scale[(size_t)h * job.scale_head_stride + tile] = __int_as_float((127 + e) << 23);
+    for (int i = 0; i < kRows; ++i) {
+      am2 = abs_max2(am2, v[i].x);
+      am2 = abs_max2(am2, v[i].y);
+      am2 = abs_max2(am2, v[i].z);
+      am2 = abs_max2(am2, v[i].w);
+    }
+    float amax = fmaxf(bf16_lo(am2), bf16_hi(am2));
 #pragma unroll
-  for (int i = 0; i < kRows; ++i) {
-    const int t = tile * 128 + r0 + i * (kThreads / VPR);
-    if (t < p.r.tokens)
-      job.dst[(size_t)t * job.token_stride + (size_t)h * job.head_stride + j] =
-          make_uint2(quant4(v[i].x, v[i].y, inv), quant4(v[i].z, v[i].w, inv));
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) s_max[g & 1][threadIdx.x >> 5] = amax;
+    __syncthreads();                               // one barrier per head: the partial maxima alternate between two rows
+    amax = s_max[g & 1][threadIdx.x & (kWarps - 1)];
+#pragma unroll
+    for (int o = kWarps / 2; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const int e = tile_scale_exponent(amax);
+    const float inv = __int_as_float((127 - e) << 23);          // 2^-e, exact; -e is in [-120, 126]
+    if (threadIdx.x == 0) job.scale[(size_t)h * job.scale_head_stride + tile] = __int_as_float((127 + e) << 23);
+#pragma unroll
+    for (int i = 0; i < kRows; ++i) {
+      const int t = t0 + i * kRowStep;
+      if (t < p.r.tokens)
+        job.dst[(size_t)t * job.token_stride + (size_t)h * job.head_stride + j] =
+            make_uint2(quant4(v[i].x, v[i].y, inv), quant4(v[i].z, v[i].w, inv));
+    }
+    if constexpr (!ROPE) {
+#pragma unroll
+      for (int i = 0; i < kRows; ++i) v[i] = nxt[i];
+    }
   }
 }
 
 int launch_tile_quant(const TileQuantParams& p, int njobs, cudaStream_t stream) {
   const int tiles = sdvg::scale_tiles(p.r.tokens);
-  if (p.r.heads > 65535 || njobs > kMaxJobs) return SDVG_ERR_BAD_SHAPE;
-  tile_quant_kernel<<<dim3(tiles, p.r.heads, njobs), kThreads, 0, stream>>>(p);
+  const int groups = (p.r.heads + kTileHeads - 1) / kTileHeads;
+  if (groups > 65535 || njobs > kMaxJobs) return SDVG_ERR_BAD_SHAPE;
+  bool rope = false;
+  for (int i = 0; i < njobs; ++i) rope = rope || p.job[i].rope;
+  const dim3 grid(tiles, groups, njobs);
+  if (rope) tile_quant_kernel<true><<<grid, kTileThreads, 0, stream>>>(p);
+  else tile_quant_kernel<false><<<grid, kTileThreads, 0, stream>>>(p);
   return sdvg::cuda_status(cudaGetLastError());
 }
 

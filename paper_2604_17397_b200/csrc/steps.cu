@@ -73,4 +73,30 @@ int sdvg_block_steps_e4m3(int steps, sdvg_cache* cache, const void* const* q, co
   return SDVG_OK;
 }
 
+int sdvg_block_steps_e4m3_tiled(int steps, sdvg_cache* cache, const void* const* q, const void* const* k,
+                                const void* const* v, void* const* q8_roped, float* const* q_tile_scale,
+                                void* const* out, int frames, int grid_h, int grid_w, int frame_offset,
+                                const float* cos_sin_tab, int tab_frames, int64_t block_index, float scale,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  SDVG_RANGE();
+  int st = check_steps(steps, cache, q, k, v, q8_roped, out, block_index, workspace, workspace_bytes, scale, 1);
+  if (st != SDVG_OK) return st;
+  if (!q_tile_scale) return SDVG_ERR_INVALID_ARG;
+  if (!cache->k_tile_scale || !cache->v_tile_scale) return SDVG_ERR_BAD_STATE;
+  if (cache->slots > 16) return SDVG_ERR_BAD_SHAPE;
+  for (int s = 0; s < steps; ++s) {
+    if (!q_tile_scale[s]) return SDVG_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(q_tile_scale[s]) & 3) return SDVG_ERR_MISALIGNED;
+  }
+  for (int s = 0; s < steps; ++s) {
+    st = sdvg_rope3d_qk_commit_e4m3_tiled(cache, q[s], k[s], v[s], q8_roped[s], q_tile_scale[s], frames, grid_h, grid_w,
+                                          frame_offset, cos_sin_tab, tab_frames, block_index, SDVG_STAGE, nullptr, stream);
+    if (st != SDVG_OK) return st;
+    st = sdvg_block_attn_fwd_e4m3_tiled(q8_roped[s], q_tile_scale[s], cache, block_index, out[s], nullptr, scale,
+                                        workspace, workspace_bytes, stream);
+    if (st != SDVG_OK) return st;
+  }
+  return SDVG_OK;
+}
+
 }  // extern "C"

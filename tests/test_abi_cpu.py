@@ -152,4 +152,41 @@ def test_e4m3_entry_points_validate_on_the_host(lib):
     assert q(0x1000, sc, 0x2000, 0, 2, 128, None) == api.SDVG_ERR_BAD_SHAPE
     assert q(0x1000, None, 0x2000, 16, 2, 128, None) == api.SDVG_ERR_INVALID_ARG
     assert q(0x1008, sc, 0x2000, 16, 2, 128, None) == api.SDVG_ERR_MISALIGNED
+    # ---- tile scales: one power-of-two scale per tile of 128 tokens and head
+    assert lib.sdvg_cache_tile_scale_floats(7, 40, 4680) == 7 * 40 * 37
+    assert lib.sdvg_cache_tile_scale_floats(7, 40, 128) == 7 * 40 and lib.sdvg_cache_tile_scale_floats(7, 40, 129) == 7 * 40 * 2
+    assert lib.sdvg_cache_tile_scale_floats(0, 40, 4680) == 0
+    commit_t, fused_t, attn_t = lib.sdvg_kv_commit_e4m3_tiled, lib.sdvg_rope3d_qk_commit_e4m3_tiled, lib.sdvg_block_attn_fwd_e4m3_tiled
+    # no scale arrays attached yet
+    assert commit_t(h8, 0x30000, 0x40000, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_BAD_STATE
+    assert attn_t(0x50000, sc, h8, 0, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_STATE
+    assert lib.sdvg_cache_set_tile_scales(h16, sc, sc) == api.SDVG_ERR_BAD_SHAPE
+    assert lib.sdvg_cache_set_tile_scales(h8, sc, None) == api.SDVG_ERR_INVALID_ARG
+    assert lib.sdvg_cache_set_tile_scales(h8, sc + 2, sc) == api.SDVG_ERR_MISALIGNED
+    assert lib.sdvg_cache_set_tile_scales(h8, sc, sc + 0x1000) == api.SDVG_OK
+    assert commit_t(h16, 0x30000, 0x40000, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert commit_t(h8, 0x30000, 0x40000, 1, api.SDVG_FINAL, None, None) == api.SDVG_ERR_BAD_STATE
+    assert commit_t(h8, 0x30000, None, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert commit_t(h8, 0x30008, 0x40000, 0, api.SDVG_FINAL, None, None) == api.SDVG_ERR_MISALIGNED
+    assert fused_t(h8, 0x50000, 0x30000, 0x40000, 0x60000, None, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert fused_t(h8, 0x50000, 0x30000, 0x40000, None, sc, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_INVALID_ARG
+    assert fused_t(h8, None, 0x30000, 0x40000, None, None, 1, 8, 7, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert fused_t(h8, None, 0x30000, 0x40000, None, None, 1, 8, 8, 0, tab, 4, 2, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_STATE
+    assert fused_t(h16, None, 0x30000, 0x40000, None, None, 1, 8, 8, 0, tab, 4, 0, api.SDVG_STAGE, None, None) == api.SDVG_ERR_BAD_SHAPE
+    assert attn_t(0x50000, sc, h8, 0, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_STATE     # block 0 not staged
+    assert attn_t(0x50000, None, h8, 0, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_INVALID_ARG
+    assert attn_t(0x50000, sc, h16, 0, 0x60000, None, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_SHAPE
+    assert attn_t(0x50000, sc, h8, 0, 0x60000, None, 0.125, 0x70010, ws, None) == api.SDVG_ERR_MISALIGNED
+    assert attn_t(0x50000, sc, h8, 0, 0x60000, None, -1.0, 0x70000, ws, None) == api.SDVG_ERR_INVALID_ARG
+    qt = lib.sdvg_quant_e4m3_tiled
+    assert qt(0x1000, 0x2000, sc, 16, 2, 64, None) == api.SDVG_ERR_BAD_SHAPE
+    assert qt(0x1000, 0x2000, None, 16, 2, 128, None) == api.SDVG_ERR_INVALID_ARG
+    assert qt(0x1000, 0x2008, sc, 16, 2, 128, None) == api.SDVG_ERR_MISALIGNED
+    PP = C.c_void_p * 2
+    two = PP(0x30000, 0x40000)
+    steps_t = lib.sdvg_block_steps_e4m3_tiled
+    assert steps_t(2, h8, two, two, two, two, None, two, 1, 8, 8, 0, tab, 4, 0, 0.125, 0x70000, ws, None) == api.SDVG_ERR_INVALID_ARG
+    assert steps_t(0, h8, two, two, two, two, two, two, 1, 8, 8, 0, tab, 4, 0, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_SHAPE
+    assert steps_t(2, h16, two, two, two, two, two, two, 1, 8, 8, 0, tab, 4, 0, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_SHAPE
+    assert steps_t(2, h8, two, two, two, two, two, two, 1, 8, 8, 0, tab, 4, 1, 0.125, 0x70000, ws, None) == api.SDVG_ERR_BAD_STATE
     assert lib.sdvg_cache_destroy(h8) == 0 and lib.sdvg_cache_destroy(h16) == 0

@@ -119,3 +119,34 @@ def test_block_steps_over_an_8_bit_ring_equal_the_separate_calls():
         assert api.sdvg_block_attn_status(ws1) == api.SDVG_OK and api.sdvg_block_attn_status(ws2) == api.SDVG_OK
         for c in (one, sep):
             api.sdvg_kv_commit_e4m3(c, ks[-1], vs[-1], inv, inv, b, api.SDVG_FINAL)
+
+
+def test_block_steps_over_a_tile_scaled_ring_equal_the_separate_calls():
+    sh = synth.Shape("steps8t", heads=2, head_dim=128, frames=1, grid_h=9, grid_w=31, slots=2)     # 279 tokens: 3 tiles
+    grid = (sh.frames, sh.grid_h, sh.grid_w)
+    tabf = 3 * sh.frames
+    tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+    one, sep = (api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True, tile_scales=True) for _ in range(2))
+    ws1, ws2 = api.attn_workspace(), api.attn_workspace()
+    for b in range(3):
+        dev = [[to_dev(x) for x in step] for step in _inputs(sh, 64, b)]
+        qs, ks, vs = ([step[t] for step in dev] for t in range(3))
+        q8 = [torch.zeros(qs[0].shape, dtype=torch.uint8, device="cuda") for _ in range(STEPS)]
+        sc = [torch.zeros((sh.heads, one.tiles), device="cuda") for _ in range(STEPS)]
+        out1 = [torch.full_like(qs[0], float("nan")) for _ in range(STEPS)]
+        api.sdvg_block_steps_e4m3_tiled(one, qs, ks, vs, q8, sc, out1, grid, b * sh.frames, tab, tabf, b, sh.scale, ws1)
+        for s in range(STEPS):
+            q8b, scb, out2 = torch.zeros_like(q8[s]), torch.zeros_like(sc[s]), torch.full_like(qs[s], float("nan"))
+            api.sdvg_rope3d_qk_commit_e4m3_tiled(sep, qs[s], ks[s], vs[s], q8b, scb, grid, b * sh.frames, tab, tabf, b,
+                                                 api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd_e4m3_tiled(q8b, scb, sep, b, out2, None, sh.scale, ws2)
+            assert torch.equal(q8[s], q8b) and torch.equal(sc[s], scb) and np.array_equal(to_bits(out1[s]), to_bits(out2)), (b, s)
+            assert not torch.isnan(out2.float()).any()
+        assert api.sdvg_block_attn_status(ws1) == api.SDVG_OK and api.sdvg_block_attn_status(ws2) == api.SDVG_OK
+        for c in (one, sep):
+            api.sdvg_kv_commit_e4m3_tiled(c, ks[-1], vs[-1], b, api.SDVG_FINAL)
+        assert torch.equal(one.k_scale, sep.k_scale) and torch.equal(one.v_scale, sep.v_scale)
+    plain = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True)
+    with pytest.raises(api.SdvgError) as e:                    # no scale arrays attached: refused before anything runs
+        api.sdvg_block_steps_e4m3_tiled(plain, qs, ks, vs, q8, sc, out1, grid, 0, tab, tabf, 0, sh.scale, ws1)
+    assert e.value.status == api.SDVG_ERR_BAD_STATE
