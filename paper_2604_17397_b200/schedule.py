@@ -37,7 +37,8 @@ class ModelState:
     tab_frames: int
     scale: float
     workspace: torch.Tensor = None
-    # 8-bit ring (cache.e4m3): static inverse scales per head, device fp32 [heads]
+    # 8-bit ring (cache.e4m3): static inverse scales per head, device fp32 [heads]; a ring with tile scales
+    # (cache.tile_scales) chooses its scales itself and takes none
     q_inv_scale: torch.Tensor = None
     k_inv_scale: torch.Tensor = None
     v_inv_scale: torch.Tensor = None
@@ -48,9 +49,13 @@ class ModelState:
         shape = (self.cache.block_tokens, self.cache.heads, self.cache.head_dim)
         dev = self.table.device
         self.e4m3 = bool(getattr(self.cache, "e4m3", False))
-        if self.e4m3:
+        self.tiled = bool(getattr(self.cache, "tile_scales", False))
+        if self.tiled:
+            # scales of the roped queries of the current step, [heads][tiles], written by the fused prologue
+            self.q_tile_scale = torch.ones((self.cache.heads, self.cache.tiles), dtype=torch.float32, device=dev)
+        elif self.e4m3:
             if self.q_inv_scale is None or self.k_inv_scale is None or self.v_inv_scale is None:
-                raise ValueError("an 8-bit ring needs q, k and v inverse scales")
+                raise ValueError("an 8-bit ring with static scales needs q, k and v inverse scales")
             self.qk_descale = 1.0 / (self.q_inv_scale * self.k_inv_scale)
             self.v_descale = 1.0 / self.v_inv_scale
         # the roped queries of the current step: bf16, or E4M3 codes for an 8-bit ring
@@ -66,7 +71,12 @@ class ModelState:
 
     def stage_and_attend(self, q, k, v, block: int, q_roped, out) -> None:
         """One denoise step of `block`: fused rope (+ quantise) + stage, then attention against the ring."""
-        if self.e4m3:
+        if self.tiled:
+            api.sdvg_rope3d_qk_commit_e4m3_tiled(self.cache, q, k, v, q_roped, self.q_tile_scale, self.grid,
+                                                 block * self.frames, self.table, self.tab_frames, block, api.SDVG_STAGE)
+            api.sdvg_block_attn_fwd_e4m3_tiled(q_roped, self.q_tile_scale, self.cache, block, out, None, self.scale,
+                                               self.workspace)
+        elif self.e4m3:
             api.sdvg_rope3d_qk_commit_e4m3(self.cache, q, k, v, q_roped, self.q_inv_scale, self.k_inv_scale,
                                            self.v_inv_scale, self.grid, block * self.frames, self.table,
                                            self.tab_frames, block, api.SDVG_STAGE)
@@ -79,7 +89,13 @@ class ModelState:
 
     def block_steps(self, qs, ks, vs, block: int, q_ropeds, outs) -> None:
         """All denoise steps of `block` in ONE library call (per step: fused rope (+ quantise) + stage, attention)."""
-        if self.e4m3:
+        if self.tiled:
+            if getattr(self, "_step_scales", None) is None or len(self._step_scales) != len(qs):
+                self._step_scales = [torch.ones_like(self.q_tile_scale) for _ in qs]
+            api.sdvg_block_steps_e4m3_tiled(self.cache, qs, ks, vs, q_ropeds, self._step_scales, outs, self.grid,
+                                            block * self.frames, self.table, self.tab_frames, block, self.scale,
+                                            self.workspace)
+        elif self.e4m3:
             api.sdvg_block_steps_e4m3(self.cache, qs, ks, vs, q_ropeds, outs, self.q_inv_scale, self.k_inv_scale,
                                       self.v_inv_scale, self.qk_descale, self.v_descale, self.grid, block * self.frames,
                                       self.table, self.tab_frames, block, self.scale, self.workspace)
@@ -96,6 +112,10 @@ class ModelState:
 
     def commit_final(self, k, v, block: int) -> int:
         """Rope the block's final K and write it with V into the ring (SDVG_FINAL); returns the evicted block."""
+        if self.tiled:
+            return api.sdvg_rope3d_qk_commit_e4m3_tiled(self.cache, None, k, v, None, None, self.grid,
+                                                        block * self.frames, self.table, self.tab_frames, block,
+                                                        api.SDVG_FINAL)
         if self.e4m3:
             return api.sdvg_rope3d_qk_commit_e4m3(self.cache, None, k, v, None, None, self.k_inv_scale, self.v_inv_scale,
                                                   self.grid, block * self.frames, self.table, self.tab_frames, block,

@@ -403,3 +403,106 @@ def test_whole_path_error_does_not_depend_on_the_magnitude_the_data_arrives_with
     moved = whole_path_errors(2.0 ** -6, 2.0 ** 6, 2.0 ** -11)
     assert abs(moved["tiled"] - unit["tiled"]) <= 1e-3, (unit, moved)
     assert moved["static"] >= 0.5, moved
+
+
+def test_schedule_with_tile_scaled_rings_follows_the_flow_and_holds_the_oracle_codes_and_scales():
+    from paper_2604_17397_b200 import schedule
+    from test_gpu_schedule import Provider
+
+    sh_d = synth.Shape("d8t", heads=3, head_dim=128, frames=3, grid_h=4, grid_w=13, slots=3)      # 156 tokens: 2 tiles
+    sh_t = synth.Shape("t8t", heads=5, head_dim=128, frames=3, grid_h=4, grid_w=13, slots=4)
+    B, steps, tau, seed = 9, 2, -0.7, 61
+    tabf = B * sh_t.frames
+    scores = synth.calibrated_scores(B, 12, seed)
+    prov = Provider(sh_d, sh_t, seed)
+    models = {}
+    for name, sh in (("drafter", sh_d), ("target", sh_t)):
+        cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True, tile_scales=True)
+        tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+        models[name] = schedule.ModelState(cache, (sh.frames, sh.grid_h, sh.grid_w), tab, tabf, sh.scale)
+    shapes = {"drafter": sh_d, "target": sh_t}
+    checked = []
+
+    def on_attention(model, b, s, q8, out):
+        if (b + s) % 3:
+            return
+        m, sh = models[model], shapes[model]
+        T = sh.block_tokens
+        ks, vs, ksc, vsc = [], [], [], []
+        for blk in range(max(0, b - (sh.slots - 1)), b + 1):       # the window as the device ring holds it now
+            slot = blk % sh.slots
+            gk, gv = m.cache.read_block(slot)
+            ks.append(gk.cpu().numpy())
+            vs.append(gv.cpu().numpy())
+            ksc.append(O.e4m3_token_scales(m.cache.k_scale[:, slot].cpu().numpy(), T))
+            vsc.append(O.e4m3_token_scales(m.cache.v_scale[:, slot].cpu().numpy(), T))
+        k_all, v_all, ksc, vsc = np.concatenate(ks), np.concatenate(vs), np.concatenate(ksc), np.concatenate(vsc)
+        qsc = O.e4m3_token_scales(m.q_tile_scale.cpu().numpy(), T)
+        r = np.random.default_rng([seed, b, s])
+        h = int(r.integers(sh.heads))
+        rows = np.sort(r.choice(T, 16, replace=False))
+        q8n = q8.cpu().numpy()
+        o_ref, _ = O.attn_e4m3_rowscaled_ref(q8n, qsc, k_all, ksc, v_all, vsc, sh.scale, heads=[h], rows=rows)
+        qd = O.e4m3_decode(q8n) * qsc[:, :, None]
+        kd = O.e4m3_decode(k_all) * ksc[:, :, None]
+        vd = O.e4m3_decode(v_all) * vsc[:, :, None]
+        bound = p_rounding_bound_tiled(qd, kd, vd, vsc[:, h], sh.scale, h, rows)
+        check_attention(out[torch.from_numpy(rows).cuda(), h], o_ref[:, 0], bound, (model, b, s))
+        checked.append((model, b, s))
+
+    res = schedule.run_schedule(B, steps, torch.from_numpy(scores).cuda(), tau, models["drafter"], models["target"],
+                                prov.device, on_attention=on_attention)
+    for m in models.values():
+        assert api.sdvg_block_attn_status(m.workspace) == api.SDVG_OK
+    assert len(checked) >= 6 and {c[0] for c in checked} == {"drafter", "target"}
+    # the flow is that of the oracle's schedule; its bf16 rings, quantised tile by tile, are what the rings must hold
+    rd = O.RingCacheRef(sh_d.slots, sh_d.heads, sh_d.block_tokens, sh_d.head_dim)
+    rt = O.RingCacheRef(sh_t.slots, sh_t.heads, sh_t.block_tokens, sh_t.head_dim)
+    want = O.schedule_ref(B, steps, scores, tau, rd, rt, prov.bits, (sh_d.frames, sh_d.grid_h, sh_d.grid_w),
+                          (sh_t.frames, sh_t.grid_h, sh_t.grid_w), sh_t.frames,
+                          O.rope_table(128, tabf, sh_d.grid_h, sh_d.grid_w), O.rope_table(128, tabf, sh_t.grid_h, sh_t.grid_w),
+                          tabf)
+    assert np.array_equal(res.accept, want.accept) and res.target_source == want.target_source
+    assert res.drafter_evicted == want.drafter_evicted and res.target_evicted == want.target_evicted
+    assert res.drafter_attn_calls == want.drafter_attn_calls and res.target_attn_calls == want.target_attn_calls
+    for name, ref in (("drafter", rd), ("target", rt)):
+        cache = models[name].cache
+        assert cache.state()[:2] == (ref.next_block, ref.slot_block)
+        for s in range(ref.slots):
+            gk, gv = cache.read_block(s)
+            k8, ks = O.quant_e4m3_tiled_ref(ref.k[s])
+            v8, vs = O.quant_e4m3_tiled_ref(ref.v[s])
+            assert np.array_equal(gk.cpu().numpy(), k8) and np.array_equal(gv.cpu().numpy(), v8), (name, s)
+            assert np.array_equal(cache.k_scale[:, s].cpu().numpy(), ks) and np.array_equal(cache.v_scale[:, s].cpu().numpy(), vs)
+        cache.close()
+
+
+def test_block_steps_of_a_tile_scaled_ring_replayed_from_a_cuda_graph_equal_the_eager_calls():
+    from paper_2604_17397_b200 import schedule
+
+    sh = synth.Shape("graph8t", heads=3, head_dim=128, frames=3, grid_h=6, grid_w=11, slots=3)
+    tabf, steps = 4 * sh.frames, 3
+    cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, e4m3=True, tile_scales=True)
+    tab = api.sdvg_rope3d_table(sh.head_dim, tabf, sh.grid_h, sh.grid_w).cuda()
+    m = schedule.ModelState(cache, (sh.frames, sh.grid_h, sh.grid_w), tab, tabf, sh.scale)
+    for b in range(3):                                  # block 2 sees two committed blocks
+        if b == 2:
+            g = schedule.BlockStepGraph(m, b, steps)
+            eager, eager_q8 = [], []
+            for s in range(steps):
+                q, k, v = (to_dev(synth.block_tensor(sh, 98, b, s, t)) for t in (synth.Q, synth.K, synth.V))
+                g.q[s].copy_(q); g.k[s].copy_(k); g.v[s].copy_(v)
+                m.stage_and_attend(q, k, v, b, m.q_roped, m.out)
+                eager.append(m.out.clone())
+                eager_q8.append(m.q_roped.clone())
+            for o in g.out:
+                o.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            assert api.sdvg_block_attn_status(m.workspace) == api.SDVG_OK
+            for s in range(steps):
+                assert torch.equal(g.q_roped[s], eager_q8[s]), s
+                assert torch.equal(g.out[s].view(torch.int16), eager[s].view(torch.int16)), s
+        k, v = (to_dev(synth.block_tensor(sh, 98, b, 9, t)) for t in (synth.K, synth.V))
+        m.commit_final(k, v, b)
+    cache.close()
