@@ -201,7 +201,10 @@ int sdvg_block_attn_fwd(const void* q, const void* k_self, const void* v_self,
  * NULL entries).  All caches must have the same block_tokens, heads and head_dim.  Problems whose visible
  * key segments agree (same ring fill, same staging: the normal case) are processed by ONE launch whose
  * work items span all problems, which is what fills the GPU at the drafter's shape; otherwise the
- * problems are launched one after the other on `stream`.  Results are those of `batch` separate calls.
+ * problems are launched one after the other on `stream`.  Results are those of `batch` separate calls up to
+ * the order of one summation: how a launch deals its query tiles to the SMs depends on how many tiles it has, and a
+ * tile is either processed whole or with its keys split into two partial results that are merged at the end.
+ * Where both launches treat a tile alike (always when neither has more than two tiles per SM) the bits agree.
  * Errors: those of sdvg_block_attn_fwd; BAD_SHAPE for batch > 4 or mismatched cache shapes.
  */
 int sdvg_block_attn_fwd_batched(int batch, const void* const* q, const void* const* k_self,
@@ -415,7 +418,8 @@ int sdvg_block_attn_fwd_e4m3(const void* q8, const void* k_self8, const void* v_
  * and the unconditional pass that a guidance scale of 3.0 implies, Sec. 4.1 "Models"), each with its own ring
  * and its own scale vectors, in one launch when their key segments agree (else one launch each, in stream
  * order).  All arrays are HOST arrays of `batch` entries; k_self8 / v_self8 / lse may be NULL (not given for
- * any problem) or hold NULL entries.  Results equal those of separate sdvg_block_attn_fwd_e4m3 calls, bit for bit.
+ * any problem) or hold NULL entries.  Results are those of separate sdvg_block_attn_fwd_e4m3 calls (see
+ * sdvg_block_attn_fwd_batched for what "those" means).
  */
 int sdvg_block_attn_fwd_e4m3_batched(int batch, const void* const* q8, const void* const* k_self8,
                                      const void* const* v_self8, const sdvg_cache* const* caches,

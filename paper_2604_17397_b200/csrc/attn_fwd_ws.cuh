@@ -1,8 +1,7 @@
 // Warp-specialised, persistent block-attention kernel (included by attn_fwd.cu after the common
-// definitions).  One CTA of 20 warps per SM; a work item is a pair of 128-row query tiles ("lanes").
-// Usually the two tiles belong to one head and share every K/V tile; a pair that straddles a head
-// boundary has lanes that stream their own K/V, and the tiles left over after the pairs run alone,
-// their keys split between the two lanes.
+// definitions).  One CTA of 20 warps per SM; a work item is a pair of 128-row query tiles ("lanes") of one
+// head, which share every K/V tile, or a single tile whose keys are split between the two lanes
+// (attn_schedule.h says which CTA gets which).
 //
 //   warps 0-3    softmax of lane 0, key columns 0-63 of every tile     \  two threads per query row: a warp
 //   warps 4-7    softmax of lane 1, key columns 0-63                    \ reaches the 32 TMEM lanes of its place
@@ -45,6 +44,8 @@
 // scales enter as a factor of the logit scale and of the final 1/l.  Everything else is shared.
 #pragma once
 
+#include "attn_schedule.h"
+
 
 // F8: operands are E4M3 bytes instead of bf16 (a row of 128 dims is then one 128-byte panel).
 template <int D, bool F8 = false>
@@ -75,55 +76,6 @@ struct WsCfg {
   static_assert(5 * 32 * kLaunchRegs <= 16384, "register file of a sub-partition");
   static_assert(4 * kSoftmaxRegs + kIssueRegs <= 5 * kLaunchRegs, "register pool of a sub-partition");
   static_assert(kDynamic <= 232448, "shared memory budget");
-};
-
-struct WsItem {
-  int head[2], tile[2];   // per lane
-  int lanes;              // 1 or 2
-  bool dual;              // lanes stream their own K/V tiles (different heads, or one tile split by keys)
-  bool split;             // both lanes work on ONE query tile: lane i takes key tiles i, i + 2, i + 4, ...
-  int nk[2];              // key tiles per lane
-  // branch-free on purpose: a loop-invariant branch on `split` makes the compiler clone whole role loops
-  __device__ int key_tile(int lane, int t) const { return (t << (int)split) + (lane & -(int)split); }
-};
-
-// Static schedule.  The query tiles of all heads form one list (head-major); with G CTAs and U tiles,
-// the first P = G * floor(U / 2G) items are pairs of neighbouring tiles (tiles 2v and 2v+1: the same
-// head, or, where the pair straddles a head boundary, two heads whose lanes stream their own K/V),
-// the remaining U - 2P tiles are items of one tile each, whose keys are split between the two lanes
-// (even and odd key tiles; the two partial results are merged when the item ends), so that a single
-// tile costs about half a pair.  Items are dealt round-robin, so every CTA gets the same number of
-// pairs, CTAs that run at the same time work on neighbouring tiles of few heads (their K/V tiles are
-// shared through L2), and the single tiles even out the last round.
-struct WsSchedule {
-  int tiles, num_pairs, num_items;
-  __host__ __device__ WsSchedule(int tokens, int heads, int ctas) {
-    tiles = (tokens + kTileM - 1) / kTileM;
-    const int total = tiles * heads;
-    num_pairs = (total / (2 * ctas)) * ctas;
-    num_items = num_pairs + (total - 2 * num_pairs);
-  }
-  __device__ void get(int v, int ntiles_k, WsItem& it) const {
-    const int g0 = v < num_pairs ? 2 * v : 2 * num_pairs + (v - num_pairs);
-    it.head[0] = g0 / tiles;
-    it.tile[0] = g0 - it.head[0] * tiles;
-    if (v < num_pairs) {
-      it.head[1] = (g0 + 1) / tiles;
-      it.tile[1] = g0 + 1 - it.head[1] * tiles;
-      it.lanes = 2;
-      it.dual = it.head[1] != it.head[0];
-      it.split = false;
-      it.nk[0] = it.nk[1] = ntiles_k;
-    } else {
-      it.head[1] = it.head[0];
-      it.tile[1] = it.tile[0];
-      it.split = ntiles_k >= 2;
-      it.lanes = it.split ? 2 : 1;
-      it.dual = true;
-      it.nk[0] = it.split ? (ntiles_k + 1) / 2 : ntiles_k;
-      it.nk[1] = it.split ? ntiles_k / 2 : 0;
-    }
-  }
 };
 
 // Ring position (stage, phase parity) advanced one stage at a time.
@@ -372,7 +324,7 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
   // Every wait of this kernel gives up at the same absolute time; a thread that gives up records
   // the timeout and leaves its role loop, and all roles meet at the common exit below.
   const Deadline dl{globaltimer_ns() + kWaitLimitNs, p.work + 1};
-  const WsSchedule sched(p.tokens, p.heads * p.batch, gridDim.x);   // it.head[] are global heads: problem * heads + head
+  const WsSchedule sched(p.tokens, p.heads * p.batch, gridDim.x, kTileM);   // it.head[] are global heads: problem * heads + head
   int ntiles_k = 0;
   if constexpr (TS) ntiles_k = p.ts_nslots * p.ts_tiles;
   else
@@ -423,10 +375,9 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         ++kv_issued;
       };
 
+      WsItem it;
       #pragma unroll 1
-      for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
-        WsItem it;
-        sched.get(v, ntiles_k, it);
+      for (int n = 0; alive && sched.get(blockIdx.x, n, ntiles_k, it); ++n) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           if (i >= it.lanes || !alive) break;
@@ -504,10 +455,9 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
         }
       };
 
+      WsItem it;
       #pragma unroll 1
-      for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
-        WsItem it;
-        sched.get(v, ntiles_k, it);
+      for (int n = 0; alive && sched.get(blockIdx.x, n, ntiles_k, it); ++n) {
         const int nl = it.lanes;
         const bool dual = it.dual;
         const int nk0 = it.nk[0], nk1 = it.nk[1];      // scalars: indexing the item by the lane would put it in local memory
@@ -547,10 +497,9 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       const uint64_t descV0 = smem_desc_sw128(sKV, C::kPanelBytes, 1024);
       constexpr int kSlices = F8 ? 4 : 8;  // MMAs per key tile: 32 or 16 keys each
 
+      WsItem it;
       #pragma unroll 1
-      for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
-        WsItem it;
-        sched.get(v, ntiles_k, it);
+      for (int n = 0; alive && sched.get(blockIdx.x, n, ntiles_k, it); ++n) {
         const int nl = it.lanes;
         const bool dual = it.dual;
         const int nk0 = it.nk[0], nk1 = it.nk[1];
@@ -613,10 +562,9 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
     uint64_t c2x2 = pack2(c2, c2);
     uint32_t s_cnt = 0, pv_cnt = 0, item_cnt = 0, split_cnt = 0;
     bool alive = true;
+    WsItem it;
     #pragma unroll 1
-    for (int v = blockIdx.x; v < sched.num_items && alive; v += gridDim.x) {
-      WsItem it;
-      sched.get(v, ntiles_k, it);
+    for (int n = 0; alive && sched.get(blockIdx.x, n, ntiles_k, it); ++n) {
       if (it.lanes <= i) continue;
       // this lane's fields as scalars (indexing the item by the lane would put it in local memory)
       const int my_nk = i == 0 ? it.nk[0] : it.nk[1];
