@@ -1,7 +1,8 @@
 // Warp-specialised, persistent block-attention kernel (included by attn_fwd.cu after the common
-// definitions).  One CTA of 20 warps per SM; a work item is a pair of 128-row query tiles ("lanes") of one
-// head, which share every K/V tile, or a single tile whose keys are split between the two lanes
-// (attn_schedule.h says which CTA gets which).
+// definitions).  One CTA of 20 warps per SM; a work item is a pair of 128-row query tiles ("lanes").
+// Usually the two tiles belong to one head and share every K/V tile; a pair that straddles a head
+// boundary has lanes that stream their own K/V, and the tiles left over after the pairs run alone,
+// their keys split between the two lanes (attn_schedule.h says which CTA gets which).
 //
 //   warps 0-3    softmax of lane 0, key columns 0-63 of every tile     \  two threads per query row: a warp
 //   warps 4-7    softmax of lane 1, key columns 0-63                    \ reaches the 32 TMEM lanes of its place
