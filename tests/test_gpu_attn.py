@@ -108,6 +108,14 @@ def test_closed_forms_on_device():
     assert np.allclose(lse.cpu().numpy(), np.log(sh.block_tokens), atol=1e-4)
 
 
+def rows_touching_every_tile(rng, tokens, extra):
+    """One random row of every 128-row query tile plus `extra` random rows: no tile of a head goes unsampled."""
+    tiles = (tokens + 127) // 128
+    one_each = [int(rng.integers(t * 128, min(tokens, (t + 1) * 128))) for t in range(tiles)]
+    more = rng.choice(tokens, extra, replace=False)
+    return np.unique(np.concatenate([one_each, more]))
+
+
 def test_config2_wan13b_shape_sampled_and_two_full_heads():
     sh = synth.WAN_1_3B
     cache = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim)
@@ -119,14 +127,15 @@ def test_config2_wan13b_shape_sampled_and_two_full_heads():
         api.sdvg_kv_commit(cache, to_dev(k), to_dev(v), b, api.SDVG_FINAL)
         ref.commit(b, k, v, O.FINAL)
     q, k, v = (synth.block_tensor(sh, 2, 2, 0, t) for t in (synth.Q, synth.K, synth.V))
-    out = torch.empty_like(to_dev(q))
+    out = torch.full_like(to_dev(q), float("nan"))
     api.sdvg_kv_commit(cache, to_dev(k), to_dev(v), 2, api.SDVG_STAGE)
     api.sdvg_block_attn_fwd(to_dev(q), None, None, cache, 2, out, None, sh.scale, ws)
     assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    assert not torch.isnan(out.float()).any()                  # every row of every tile was written
     got = to_bits(out)
     rng = np.random.default_rng(2)
     for h in range(sh.heads):
-        rows = np.arange(sh.block_tokens) if h in (0, 11) else np.sort(rng.choice(sh.block_tokens, 96, replace=False))
+        rows = np.arange(sh.block_tokens) if h in (0, 11) else rows_touching_every_tile(rng, sh.block_tokens, 64)
         o_ref, _ = O.block_attn_ref(q, k, v, ref, 2, sh.scale, heads=[h], rows=rows)
         check(got[rows, h], o_ref[:, 0], ("wan1.3b", h))
 
@@ -153,10 +162,11 @@ def test_config3_wan14b_shape_fused_prologue_cache_bits_and_sampled_attention():
     q_r = torch.empty_like(dq)
     api.sdvg_rope3d_qk_commit(cache, dq, to_dev(k), to_dev(v), q_r, None, grid, b * sh.frames, dev_tab, tabf, b,
                               api.SDVG_STAGE)
-    out = torch.empty_like(dq)
-    lse = torch.empty((sh.heads, sh.block_tokens), device="cuda")
+    out = torch.full_like(dq, float("nan"))
+    lse = torch.full((sh.heads, sh.block_tokens), float("nan"), device="cuda")
     api.sdvg_block_attn_fwd(q_r, None, None, cache, b, out, lse, sh.scale, ws)
     assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    assert not torch.isnan(out.float()).any() and not torch.isnan(lse).any()      # every row of every tile was written
     qr_ref = O.rope_bitspec(q, grid, b * sh.frames, ref_tab, tabf)
     kr_ref = O.rope_bitspec(k, grid, b * sh.frames, ref_tab, tabf)
     assert np.array_equal(to_bits(q_r), qr_ref)
@@ -170,7 +180,7 @@ def test_config3_wan14b_shape_fused_prologue_cache_bits_and_sampled_attention():
     rng = np.random.default_rng(3)
     lse_h = lse.cpu().numpy()
     for h in range(sh.heads):
-        rows = np.arange(sh.block_tokens) if h in (0, 39) else np.sort(rng.choice(sh.block_tokens, 64, replace=False))
+        rows = np.arange(sh.block_tokens) if h in (0, 39) else rows_touching_every_tile(rng, sh.block_tokens, 30)
         o_ref, lse_ref = O.block_attn_ref(qr_ref, kr_ref, v, ref, b, sh.scale, heads=[h], rows=rows)
         check(got[rows, h], o_ref[:, 0], ("wan14b", h))
         assert np.allclose(lse_h[h, rows], lse_ref[0], rtol=0, atol=2e-3)
