@@ -322,3 +322,36 @@ def test_smallest_rings(slots, staged):
     # slots = 1: a block sees only itself; slots = 2: itself and the block before it
     sh = synth.Shape(f"ring{slots}", heads=2, head_dim=64, frames=1, grid_h=9, grid_w=17, slots=slots)
     run_sequence(sh, 4, 95 + slots, staged)
+
+
+def test_several_rounds_of_pairs_with_odd_tiles_per_head_single_and_batched():
+    # 41 heads x 15 tiles = 615 tiles: on a 148-SM GPU two full rounds of pairs (dealt one CTA further on in the
+    # second round), pairs that straddle heads in both, 23 key-split singles; two problems in one call double that.
+    # Every head is checked on a row of every one of its tiles.
+    sh = synth.Shape("rounds", heads=41, head_dim=128, frames=1, grid_h=38, grid_w=50, slots=2)      # 1900 tokens
+    caches = [api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim) for _ in range(2)]
+    refs = [O.RingCacheRef(sh.slots, sh.heads, sh.block_tokens, sh.head_dim) for _ in range(2)]
+    ws = api.attn_workspace()
+    rng = np.random.default_rng(17)
+    for n in range(2):
+        k0, v0 = synth.block_tensor(sh, 90 + n, 0, 0, synth.K), synth.block_tensor(sh, 90 + n, 0, 0, synth.V)
+        api.sdvg_kv_commit(caches[n], to_dev(k0), to_dev(v0), 0, api.SDVG_FINAL)
+        refs[n].commit(0, k0, v0, O.FINAL)
+    qkv = [[synth.block_tensor(sh, 90 + n, 1, 0, t) for t in (synth.Q, synth.K, synth.V)] for n in range(2)]
+    dev = [[to_dev(x) for x in prob] for prob in qkv]
+    for n in range(2):
+        api.sdvg_kv_commit(caches[n], dev[n][1], dev[n][2], 1, api.SDVG_STAGE)
+    one = torch.full_like(dev[0][0], float("nan"))
+    api.sdvg_block_attn_fwd(dev[0][0], None, None, caches[0], 1, one, None, sh.scale, ws)
+    outs = [torch.full_like(dev[n][0], float("nan")) for n in range(2)]
+    api.sdvg_block_attn_fwd_batched([d[0] for d in dev], None, None, caches, [1, 1], outs, None, sh.scale, ws)
+    assert api.sdvg_block_attn_status(ws) == api.SDVG_OK
+    for o in [one] + outs:
+        assert not torch.isnan(o.float()).any()
+    for h in range(sh.heads):
+        rows = rows_touching_every_tile(rng, sh.block_tokens, 8)
+        for n in range(2):
+            o_ref, _ = O.block_attn_ref(*qkv[n], refs[n], 1, sh.scale, heads=[h], rows=rows)
+            check(to_bits(outs[n])[rows, h], o_ref[:, 0], ("rounds batched", n, h))
+            if n == 0:
+                check(to_bits(one)[rows, h], o_ref[:, 0], ("rounds single", h))
