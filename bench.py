@@ -517,7 +517,6 @@ def e4m3_figures(st, pk, device):
     elems = sh.block_tokens * sh.heads * sh.head_dim
     a = stats(t_attn8, attn_flops(sh, st.lk), 1e-9, 2 * pk["bf16_tflops"])
     cm = stats(t_commit8, 2 * elems * 3, 1e-6, pk["hbm_gbs"])
-    c8.close()
     # the same with one power-of-two scale per tile of 128 tokens and head, chosen by the library from the data
     ct = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device, e4m3=True, tile_scales=True)
     for n in range(sh.slots - 1):
@@ -532,6 +531,25 @@ def e4m3_figures(st, pk, device):
     t_attn_t = time_launches(torch, [lambda: api.sdvg_block_attn_fwd_e4m3_tiled(q8, qs, ct, blk, st.out, None, sh.scale,
                                                                                 st.ws)])
     assert api.sdvg_block_attn_status(st.ws) == api.SDVG_OK
+    # The three attention kernels in the SAME power state: bf16, 8-bit with static scales and 8-bit with tile scales,
+    # alternately, two launches at a time (figures taken minutes apart in a long run differ by more than the kernels do).
+    cb = api.Cache(sh.slots, sh.heads, sh.block_tokens, sh.head_dim, device=device)
+    for n in range(sh.slots - 1):
+        api.sdvg_kv_commit(cb, st.k_r, st.v, n, api.SDVG_FINAL)
+    api.sdvg_kv_commit(cb, st.k_r, st.v, blk, api.SDVG_STAGE)
+    trio = {"bf16": lambda: api.sdvg_block_attn_fwd(st.q_r, None, None, cb, blk, st.out, None, sh.scale, st.ws),
+            "e4m3": lambda: api.sdvg_block_attn_fwd_e4m3(q8, None, None, c8, blk, qk_desc, desc, st.out, None, sh.scale,
+                                                         st.ws),
+            "e4m3_tiled": lambda: api.sdvg_block_attn_fwd_e4m3_tiled(q8, qs, ct, blk, st.out, None, sh.scale, st.ws)}
+    side = {k: [] for k in trio}
+    names = list(trio)
+    for i in range(3 * (TIMED_LAUNCHES // 6 + 1)):            # every order of succession equally often
+        for j in range(3):
+            k = names[(i + j * (1 + i // 3 % 2)) % 3]
+            side[k] += time_launches(torch, [trio[k]], n=2, warm=0)
+    side = {k: float(np.median(v)) for k, v in side.items()}
+    cb.close()
+    c8.close()
     at = stats(t_attn_t, attn_flops(sh, st.lk), 1e-9, 2 * pk["bf16_tflops"])
     cmt = stats(t_commit_t, 2 * elems * 3, 1e-6, pk["hbm_gbs"])
     prt = stats(t_pro_t, 3 * elems * 3, 1e-6, pk["hbm_gbs"])
@@ -541,6 +559,9 @@ def e4m3_figures(st, pk, device):
             "peak_source": "measured bf16 burst peak x the nominal fp8/bf16 ratio of 2", "frac": a["frac"],
             "kv_commit_e4m3": {"ms_median": cm["ms_median"], "gbs": cm["rate_median"], "frac": cm["frac"]},
             "note": "operands E4M3 with one static scale per head, P rounded to E4M3",
+            "same_state_ms": {**side, "note": "the three kernels launched alternately, two launches at a time, median",
+                              "e4m3_over_bf16": side["e4m3"] / side["bf16"],
+                              "e4m3_tiled_over_bf16": side["e4m3_tiled"] / side["bf16"]},
             "tile_scales": {"kernel": "sdvg_block_attn_fwd_e4m3_tiled", "ms_median": at["ms_median"],
                             "ms_min": at["ms_min"], "tflops": at["rate_median"], "tflops_best": at["rate_best"],
                             "frac": at["frac"],

@@ -580,16 +580,22 @@ __global__ void __launch_bounds__(WsCfg<D, F8>::kThreads, 1) attn_fwd_ws_kernel(
       }
       float m_ref = -INFINITY, l_run = 0.f, neg = 0.f;     // neg = -m_ref * c2 (+ the window shift)
       int lv_ref = 0;                                      // tile scales: exponent of the V scale that O is relative to
+      // tile scales: this lane's current key tile as (visible slot, tile of the slot), stepped along with j
+      int ts_sl = 0, ts_tl = TS ? it.key_tile(i, 0) : 0;
+      const int ts_step = 1 << (int)it.split;
+      if constexpr (TS)
+        while (ts_tl >= p.ts_tiles) ts_tl -= p.ts_tiles, ++ts_sl;
       #pragma unroll 1
       for (int j = 0; j < my_nk && alive; ++j) {          // this lane's j-th key tile
         // number of real keys in that tile: the last tile of a key segment may be ragged
-        const int valid = key_tile_valid<TS>(p, it.key_tile(i, j));
+        const int valid = TS ? min(kTileN, p.tokens - ts_tl * kTileN) : key_tile_valid<TS>(p, it.key_tile(i, j));
         float k_sc = 1.f, v_sc = 1.f;                      // tile scales: this key tile's K and V scales (powers of two),
         if constexpr (TS) {                                // fetched ahead of the wait for the logits
-          const int kt = it.key_tile(i, j);
-          const int idx = (my_head * p.ts_cache_slots + p.ts_slot[kt / p.ts_tiles]) * p.ts_tiles + kt % p.ts_tiles;
+          const int idx = (my_head * p.ts_cache_slots + p.ts_slot[ts_sl]) * p.ts_tiles + ts_tl;
           k_sc = __ldg(p.prob[0].k_tile_scale + idx);
           v_sc = __ldg(p.prob[0].v_tile_scale + idx);
+          ts_tl += ts_step;
+          while (ts_tl >= p.ts_tiles) ts_tl -= p.ts_tiles, ++ts_sl;
         }
         const uint32_t par = s_cnt & 1;
         if (!(alive = wait_bar(&s_full[i], par, dl))) break;
